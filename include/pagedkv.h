@@ -1,0 +1,191 @@
+/*
+ * pagedkv.h -- C ABI of the B200 (sm_100a) paged-attention decode and KV-block swap library.
+ *
+ * The calls follow the serving model of the paper (arXiv 2602.07878): a decode step reads
+ * the KV cache of every running sequence through a logical-to-physical block map
+ * (Section 2.1 "Decoding", Section 2.2 "KV-Cache", Section 4.2 / Eq. 3), and preemption by
+ * swapping moves a victim's KV blocks to host memory and later back into newly allocated
+ * blocks (Section 5.1.2 "Swapping").
+ *
+ * Conventions for every call
+ *   - Plain C types only.  "dev" pointers are CUDA device addresses, "host" pointers are
+ *     host addresses; "pinned" means page-locked host memory that the GPU can address.
+ *   - The caller owns every buffer (inputs, outputs, workspace, staging, host images).
+ *     Unless a call's comment says otherwise the library allocates no device memory and
+ *     keeps no state besides cached device properties.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and the call returns without waiting for the GPU.
+ *   - The return value is PA_OK or a negative PA_ERR_* code for an error found on the
+ *     host; in that case nothing was launched.  Errors in device-resident data (a bad
+ *     length or block id) cannot be seen by the host without a sync; they are reported
+ *     through the optional `dev_status` word and never make the GPU read outside the pool.
+ *   - bf16 is the only element type; accumulation is fp32.
+ */
+#ifndef PAGEDKV_H_
+#define PAGEDKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- host-side return codes ---------------------------------------------------------- */
+#define PA_OK 0
+#define PA_ERR_NULL (-1)      /* a required pointer is NULL                                */
+#define PA_ERR_SHAPE (-2)     /* unsupported head_dim / block_size / head counts / strides */
+#define PA_ERR_ALIGN (-3)     /* a buffer is not 16-byte aligned                           */
+#define PA_ERR_WORKSPACE (-4) /* workspace / staging buffer too small                      */
+#define PA_ERR_HOSTBUF (-5)   /* host image buffer too small                               */
+#define PA_ERR_BLOCK_ID (-6)  /* swap block id out of range or listed twice                */
+#define PA_ERR_CUDA (-7)      /* a CUDA runtime/driver call failed; see pa_last_cuda_error */
+#define PA_ERR_ARG (-8)       /* negative count, bad partition size or similar             */
+
+/* ---- bits OR-ed into *dev_status by the kernels -------------------------------------- */
+#define PA_STATUS_BAD_SEQ_LEN 1   /* seq_lens[b] < 0 or > max_blocks_per_seq * block_size  */
+#define PA_STATUS_BAD_BLOCK_ID 2  /* a used block-table entry is outside [0, num_blocks)   */
+#define PA_STATUS_TIMEOUT 4       /* a bounded wait inside a kernel gave up                */
+#define PA_STATUS_WORKSPACE 8     /* the partition plan does not fit the workspace         */
+
+#define PA_BF16 1
+
+/* pa_decode flags */
+#define PA_FLAG_REUSE_PLAN 1 /* skip planning: workspace still holds the plan of an earlier
+                                call with the same seq_lens, batch and partition_tokens  */
+
+/*
+ * Geometry of one layer's K (and identically V) cache.  Element (block p, kv head h,
+ * slot t, dim d) lives at  base + p*stride_block + h*stride_head + t*stride_tok + d
+ * (strides in bf16 elements, dim is contiguous).  The recommended layout is
+ * [num_blocks][num_kv_heads][block_size][head_dim]; any strides that are multiples of
+ * 8 elements are accepted.
+ */
+typedef struct pa_shape {
+    int32_t num_q_heads;  /* H; a multiple of num_kv_heads, H / Hkv <= 16                  */
+    int32_t num_kv_heads; /* Hkv                                                           */
+    int32_t head_dim;     /* D: 64 or 128                                                  */
+    int32_t block_size;   /* tokens per block: 16                                          */
+    int32_t num_blocks;   /* physical pool size                                            */
+    int32_t dtype;        /* PA_BF16                                                       */
+    int64_t stride_block;
+    int64_t stride_head;
+    int64_t stride_tok;
+} pa_shape;
+
+/* All layers of a pool: layer l of K starts layer_stride_k elements after layer l-1. */
+typedef struct kv_pool_desc {
+    int32_t num_layers;
+    int32_t reserved;
+    int64_t layer_stride_k;
+    int64_t layer_stride_v;
+} kv_pool_desc;
+
+/*
+ * Bytes of device workspace pa_decode needs for batches of at most `max_batch` sequences
+ * holding at most `max_total_tokens` cached tokens in total.  `partition_tokens` is the
+ * value that will be passed to pa_decode (0 = automatic).  The workspace holds the
+ * partition plan and the fp32 partial results of sequences that are split (a2-a4 of the
+ * decode path: plan, partition attention, combine).
+ */
+int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch, int64_t max_total_tokens,
+                       int32_t partition_tokens, size_t* bytes);
+
+/*
+ * One decode-attention step over a paged KV cache (Section 2.1 / 2.2; Section 4.2, Eq. 3
+ * for the traffic it causes).  For every sequence b < batch and query head h:
+ *     out[b,h,:] = softmax_t( scale * <q[b,h,:], K[b,t,h/G,:]> ) . V[b,t,h/G,:],  t < seq_lens[b]
+ * where token t of sequence b is slot t % block_size of physical block
+ * block_tables[b][t / block_size] and G = num_q_heads / num_kv_heads.
+ *
+ *   q            dev bf16 [batch, H, D], contiguous, 16-byte aligned
+ *   k_cache      dev bf16, one layer, laid out per `shape`; v_cache likewise
+ *   block_tables dev int32 [batch, max_blocks_per_seq] row-major; entries at or beyond
+ *                ceil(seq_lens[b] / block_size) are never read
+ *   seq_lens     dev int32 [batch]; 0 gives a row of zeros
+ *   scale        softmax scale (e.g. 1/sqrt(D))
+ *   out          dev bf16 [batch, H, D], contiguous, 16-byte aligned
+ *   workspace    dev, >= pa_workspace_bytes(...), 256-byte aligned; contents are scratch
+ *   partition_tokens  0 = choose per call from the batch's total length; otherwise a
+ *                multiple of 16 in [16, 512]: sequences longer than this are split into
+ *                partitions of this many tokens that run in parallel and are merged by
+ *                log-sum-exp.  For a fixed value the result for a sequence depends on
+ *                nothing but its own tokens (bit-identical across batches and block ids).
+ *   flags        0 or PA_FLAG_REUSE_PLAN
+ *   dev_status   dev int32 or NULL.  PA_STATUS_* bits are OR-ed in (never cleared).  A
+ *                sequence with a bad length or a bad used block id gets an all-zero row;
+ *                the GPU never reads outside the pool.
+ * Slots of the last block beyond seq_lens[b] may hold anything (NaN included).
+ * Three kernels are enqueued (plan, partition attention, combine); nothing is synced.
+ */
+int pa_decode(const pa_shape* shape, const void* q, const void* k_cache, const void* v_cache,
+              const int32_t* block_tables, int32_t max_blocks_per_seq, const int32_t* seq_lens,
+              int32_t batch, float scale, void* out, void* workspace, size_t workspace_bytes,
+              int32_t partition_tokens, int32_t flags, int32_t* dev_status, void* cuda_stream);
+
+/* Bytes of device buffer pa_decode_host needs for its device copies of q, block tables,
+ * lengths and out. */
+int pa_host_io_bytes(const pa_shape* shape, int32_t max_batch, int32_t max_blocks_per_seq,
+                     size_t* bytes);
+
+/*
+ * pa_decode for a caller whose per-step tensors live in pinned host memory: copies
+ * q_host, block_tables_host and seq_lens_host to `io_buf` (dev, >= pa_host_io_bytes),
+ * runs pa_decode on the copies and copies the result to out_host, all on `cuda_stream`.
+ * The KV cache itself stays on the device.  out_host is valid once the stream has
+ * reached the end of this call.
+ */
+int pa_decode_host(const pa_shape* shape, const void* q_host, const void* k_cache,
+                   const void* v_cache, const int32_t* block_tables_host,
+                   int32_t max_blocks_per_seq, const int32_t* seq_lens_host, int32_t batch,
+                   float scale, void* out_host, void* io_buf, size_t io_bytes, void* workspace,
+                   size_t workspace_bytes, int32_t partition_tokens, int32_t* dev_status,
+                   void* cuda_stream);
+
+/* Bytes of one block's host image: num_layers * 2 * Hkv * block_size * D * 2. */
+int kv_block_bytes(const kv_pool_desc* pool, const pa_shape* shape, size_t* bytes);
+
+/*
+ * Swap-out (Section 5.1.2 "Swapping": the victim's KV blocks are offloaded from GPU
+ * memory to host memory).  Packs whole blocks -- every layer, K then V, unused slots
+ * included, bit for bit -- into a contiguous host image laid out
+ *     [i < n][layer][K|V][kv head][slot][dim]
+ * so that slot i of the image holds physical block block_ids[i].
+ *
+ *   k_pool, v_pool   dev bf16 pools holding all layers (see kv_pool_desc / pa_shape)
+ *   block_ids        HOST int32 [n]; copied before the call returns; each in
+ *                    [0, num_blocks) and listed once
+ *   pinned_host_buf  pinned host memory, 16-byte aligned, >= n * kv_block_bytes
+ *   staging          dev scratch or NULL.  With a staging buffer (any size >= one block
+ *                    image, 256-byte aligned) blocks are gathered into it by a kernel and
+ *                    moved by the copy engine in pieces of staging_bytes; with NULL the
+ *                    gather kernel stores straight into the pinned buffer.
+ * The image is complete when `cuda_stream` reaches the end of the call.
+ */
+int kv_swap_out(const kv_pool_desc* pool, const pa_shape* shape, const void* k_pool,
+                const void* v_pool, const int32_t* block_ids, int32_t n, void* pinned_host_buf,
+                size_t host_bytes, void* staging, size_t staging_bytes, void* cuda_stream);
+
+/*
+ * Swap-in (Section 5.1.2: the blocks migrate back over the host link when the victim is
+ * re-admitted, into whatever blocks the allocator hands out).  Inverse of kv_swap_out:
+ * image slot i is written to physical block block_ids[i]; no other byte of the pools
+ * changes.  Arguments as for kv_swap_out.
+ */
+int kv_swap_in(const kv_pool_desc* pool, const pa_shape* shape, void* k_pool, void* v_pool,
+               const void* pinned_host_buf, size_t host_bytes, const int32_t* block_ids,
+               int32_t n, void* staging, size_t staging_bytes, void* cuda_stream);
+
+/* Text for a PA_* return code. */
+const char* pa_status_string(int code);
+
+/* The cudaError_t / CUresult value behind the calling thread's last PA_ERR_CUDA (0 if none). */
+int pa_last_cuda_error(void);
+
+/* Number of kernels the library has launched since it was loaded (all threads). */
+int64_t pa_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PAGEDKV_H_ */

@@ -1,0 +1,212 @@
+"""Thin Python binding of libpagedkv.so: argument marshalling only.
+
+Every function has the name and the meaning of the C entry point it forwards to (see
+include/pagedkv.h).  Tensors are torch tensors used as plain device (or pinned host)
+buffers; nothing is computed here, and there is no fallback: if the CUDA library cannot be
+loaded, importing the functions' results fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpagedkv.so")
+
+PA_OK = 0
+PA_BF16 = 1
+PA_FLAG_REUSE_PLAN = 1
+PA_STATUS_BAD_SEQ_LEN = 1
+PA_STATUS_BAD_BLOCK_ID = 2
+PA_STATUS_TIMEOUT = 4
+PA_STATUS_WORKSPACE = 8
+ERR = {"NULL": -1, "SHAPE": -2, "ALIGN": -3, "WORKSPACE": -4, "HOSTBUF": -5, "BLOCK_ID": -6,
+       "CUDA": -7, "ARG": -8}
+
+EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
+           "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
+           "pa_last_cuda_error", "pa_launch_count"]
+
+
+class PaShape(ctypes.Structure):
+    _fields_ = [("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("block_size", ctypes.c_int32),
+                ("num_blocks", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("stride_block", ctypes.c_int64), ("stride_head", ctypes.c_int64),
+                ("stride_tok", ctypes.c_int64)]
+
+
+class KvPoolDesc(ctypes.Structure):
+    _fields_ = [("num_layers", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("layer_stride_k", ctypes.c_int64), ("layer_stride_v", ctypes.c_int64)]
+
+
+class PagedKVError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().pa_status_string(code).decode()
+        if code == ERR["CUDA"]:
+            msg += f" [cuda error {lib().pa_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libpagedkv.so (built in-tree by paper_2602_07878_b200.build).  No fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2602_07878_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        psz = ctypes.POINTER(ctypes.c_size_t)
+        pshape, ppool = ctypes.POINTER(PaShape), ctypes.POINTER(KvPoolDesc)
+        L.pa_workspace_bytes.argtypes = [pshape, i32, i64, i32, psz]
+        L.pa_decode.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp, sz,
+                                i32, i32, vp, vp]
+        L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
+        L.pa_decode_host.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp,
+                                     sz, vp, sz, i32, vp, vp]
+        L.kv_block_bytes.argtypes = [ppool, pshape, psz]
+        L.kv_swap_out.argtypes = [ppool, pshape, vp, vp, vp, i32, vp, sz, vp, sz, vp]
+        L.kv_swap_in.argtypes = [ppool, pshape, vp, vp, vp, sz, vp, i32, vp, sz, vp]
+        for name in ("pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
+                     "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_last_cuda_error"):
+            getattr(L, name).restype = ctypes.c_int
+        L.pa_status_string.argtypes = [ctypes.c_int]
+        L.pa_status_string.restype = ctypes.c_char_p
+        L.pa_launch_count.argtypes = []
+        L.pa_launch_count.restype = ctypes.c_int64
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, where: str):
+    if rc != PA_OK:
+        raise PagedKVError(rc, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def shape_of(k_cache: torch.Tensor, num_q_heads: int) -> PaShape:
+    """pa_shape of a cache tensor viewed as [num_blocks, num_kv_heads, block_size, head_dim]
+    (any strides over the first three axes; the last axis must be contiguous)."""
+    assert k_cache.dtype == torch.bfloat16 and k_cache.dim() == 4 and k_cache.stride(3) == 1
+    nb, hkv, bs, d = k_cache.shape
+    return PaShape(num_q_heads, hkv, d, bs, nb, PA_BF16, k_cache.stride(0), k_cache.stride(1),
+                   k_cache.stride(2))
+
+
+def pa_workspace_bytes(shape: PaShape, max_batch: int, max_total_tokens: int,
+                       partition_tokens: int = 0) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().pa_workspace_bytes(ctypes.byref(shape), max_batch, max_total_tokens,
+                                    partition_tokens, ctypes.byref(out)), "pa_workspace_bytes")
+    return int(out.value)
+
+
+def pa_decode(q, k_cache, v_cache, block_tables, seq_lens, scale, out, workspace, *,
+              partition_tokens: int = 0, flags: int = 0, dev_status=None, stream=None,
+              shape: Optional[PaShape] = None):
+    """Forward to pa_decode.  q/out [B,H,D] bf16; caches [NB,Hkv,bs,D] bf16 views of one
+    layer; block_tables int32 [B,max_blocks]; seq_lens int32 [B]; workspace uint8."""
+    if shape is None:
+        shape = shape_of(k_cache, q.shape[1])
+        assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
+    assert block_tables.dtype == torch.int32 and seq_lens.dtype == torch.int32
+    assert q.is_contiguous() and out.is_contiguous() and block_tables.is_contiguous()
+    rc = lib().pa_decode(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                         _ptr(block_tables), block_tables.shape[1] if block_tables.dim() == 2 else 0,
+                         _ptr(seq_lens), q.shape[0], float(scale), _ptr(out), _ptr(workspace),
+                         workspace.numel() * workspace.element_size(), partition_tokens, flags,
+                         _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_decode")
+    return out
+
+
+def pa_host_io_bytes(shape: PaShape, max_batch: int, max_blocks_per_seq: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().pa_host_io_bytes(ctypes.byref(shape), max_batch, max_blocks_per_seq,
+                                  ctypes.byref(out)), "pa_host_io_bytes")
+    return int(out.value)
+
+
+def pa_decode_host(q_host, k_cache, v_cache, block_tables_host, seq_lens_host, scale, out_host,
+                   io_buf, workspace, *, partition_tokens: int = 0, dev_status=None, stream=None):
+    """Forward to pa_decode_host: q / tables / lengths / out are pinned host tensors."""
+    shape = shape_of(k_cache, q_host.shape[1])
+    for t in (q_host, block_tables_host, seq_lens_host, out_host):
+        assert not t.is_cuda and t.is_contiguous()
+    rc = lib().pa_decode_host(ctypes.byref(shape), _ptr(q_host), _ptr(k_cache), _ptr(v_cache),
+                              _ptr(block_tables_host), block_tables_host.shape[1],
+                              _ptr(seq_lens_host), q_host.shape[0], float(scale), _ptr(out_host),
+                              _ptr(io_buf), io_buf.numel() * io_buf.element_size(),
+                              _ptr(workspace), workspace.numel() * workspace.element_size(),
+                              partition_tokens, _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_decode_host")
+    return out_host
+
+
+def pool_desc(k_pool: torch.Tensor, v_pool: torch.Tensor, num_q_heads: int = 0):
+    """(kv_pool_desc, pa_shape) of pools shaped [layers, NB, Hkv, bs, D]."""
+    assert k_pool.dim() == 5 and k_pool.dtype == torch.bfloat16 and k_pool.stride(4) == 1
+    assert v_pool.shape == k_pool.shape and v_pool.stride()[1:] == k_pool.stride()[1:]
+    shape = shape_of(k_pool[0], num_q_heads or k_pool.shape[2])
+    return KvPoolDesc(k_pool.shape[0], 0, k_pool.stride(0), v_pool.stride(0)), shape
+
+
+def kv_block_bytes(k_pool, v_pool) -> int:
+    pool, shape = pool_desc(k_pool, v_pool)
+    out = ctypes.c_size_t(0)
+    _check(lib().kv_block_bytes(ctypes.byref(pool), ctypes.byref(shape), ctypes.byref(out)),
+           "kv_block_bytes")
+    return int(out.value)
+
+
+def _ids(block_ids):
+    import numpy as np
+
+    a = np.ascontiguousarray(block_ids, dtype=np.int32)
+    return a, a.ctypes.data_as(ctypes.c_void_p)
+
+
+def kv_swap_out(k_pool, v_pool, block_ids, pinned_host_buf, staging=None, stream=None):
+    """Forward to kv_swap_out.  block_ids: host int32 sequence; pinned_host_buf: pinned
+    uint8 tensor; staging: optional device uint8 tensor."""
+    pool, shape = pool_desc(k_pool, v_pool)
+    ids, pids = _ids(block_ids)
+    rc = lib().kv_swap_out(ctypes.byref(pool), ctypes.byref(shape), _ptr(k_pool), _ptr(v_pool),
+                           pids, len(ids), _ptr(pinned_host_buf),
+                           pinned_host_buf.numel() * pinned_host_buf.element_size(),
+                           _ptr(staging), 0 if staging is None else staging.numel() * staging.element_size(),
+                           _stream(stream))
+    _check(rc, "kv_swap_out")
+
+
+def kv_swap_in(k_pool, v_pool, pinned_host_buf, block_ids, staging=None, stream=None):
+    """Forward to kv_swap_in (arguments as kv_swap_out)."""
+    pool, shape = pool_desc(k_pool, v_pool)
+    ids, pids = _ids(block_ids)
+    rc = lib().kv_swap_in(ctypes.byref(pool), ctypes.byref(shape), _ptr(k_pool), _ptr(v_pool),
+                          _ptr(pinned_host_buf),
+                          pinned_host_buf.numel() * pinned_host_buf.element_size(), pids, len(ids),
+                          _ptr(staging), 0 if staging is None else staging.numel() * staging.element_size(),
+                          _stream(stream))
+    _check(rc, "kv_swap_in")
+
+
+def pa_launch_count() -> int:
+    return int(lib().pa_launch_count())

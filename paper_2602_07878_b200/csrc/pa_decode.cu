@@ -1,0 +1,906 @@
+// Paged-attention decode for sm_100a: plan -> partition attention -> combine.
+//
+// Partition attention is organised around independent warps.  A warp owns a private ring
+// of shared-memory slots; one slot holds the K tile and the V tile (16 tokens x D) of one
+// KV block of one KV head, fetched by TMA (128-byte swizzle) and announced by an
+// mbarrier.  The warp walks the block table itself, keeps NSLOT-1 blocks in flight across
+// unit boundaries, and computes  S = Q K^T  and  O += P V  with warp-level bf16 MMAs whose
+// M dimension carries the query heads of the KV head's group.  A unit of work is
+// (sequence, KV head, partition of at most 512 tokens); units are handed out longest
+// first from a device-built list through an atomic counter, so a 32K-token sequence
+// becomes 64+ units that spread over the whole chip next to the short ones.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace pk {
+
+// ======================================================================================
+// plan kernel (one CTA): validate lengths, pick the partition size, list the work items
+// ======================================================================================
+constexpr int PLAN_THREADS = 1024;
+
+struct PlanParams {
+    const int32_t* seq_lens;
+    int batch;
+    int max_blocks;
+    int Hkv;
+    int forced_p;       // 0 = automatic
+    int64_t item_cap;   // records the workspace can hold
+    int total_warps;    // decode warps on the chip
+    int* hdr;
+    int2* seq_info;     // per sequence: (first partial index, partitions)
+    int4* records;      // per item: (b, tok0, ntok | flags, partial index)
+    int* status;
+};
+
+__device__ __forceinline__ int clamp_len(int L, int max_tok, bool& bad) {
+    if (L < 0 || L > max_tok) {
+        bad = true;
+        return 0;
+    }
+    return L;
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanParams p) {
+    __shared__ long long red[5][32];
+    __shared__ int s_P, s_bad;
+    __shared__ int hist[MAX_PART / BS + 1], start[MAX_PART / BS + 1], cursor[MAX_PART / BS + 1];
+    __shared__ int scan_warp[32];
+    __shared__ int s_carry;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int max_tok = p.max_blocks * BS;
+    const int cand[4] = {64, 128, 256, 512};
+
+    // ---- pass 1: item counts for each candidate partition size ------------------------
+    long long cnt[5] = {0, 0, 0, 0, 0};
+    bool bad = false;
+    for (int b = tid; b < p.batch; b += PLAN_THREADS) {
+        const int L = clamp_len(p.seq_lens[b], max_tok, bad);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) cnt[c] += (L + cand[c] - 1) / cand[c];
+        if (p.forced_p > 0) cnt[4] += (L + p.forced_p - 1) / p.forced_p;
+    }
+#pragma unroll
+    for (int c = 0; c < 5; ++c) {
+        long long v = cnt[c];
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) red[c][warp] = v;
+    }
+    if (tid == 0) s_bad = 0;
+    if (tid < MAX_PART / BS + 1) hist[tid] = 0, cursor[tid] = 0;
+    __syncthreads();
+    if (bad) s_bad = 1;
+    if (tid == 0) {
+        long long tot[5];
+        for (int c = 0; c < 5; ++c) {
+            long long v = 0;
+            for (int w = 0; w < PLAN_THREADS / 32; ++w) v += red[c][w];
+            tot[c] = v;
+        }
+        int P = 0;
+        if (p.forced_p > 0) {
+            P = tot[4] <= p.item_cap ? p.forced_p : 0;
+        } else {
+            // walk from the largest partition down: stop as soon as every warp gets several
+            // units; never take a size whose items do not fit the workspace
+            const long long want = 4LL * p.total_warps;
+            for (int c = 3; c >= 0; --c) {
+                if (tot[c] > p.item_cap) break;
+                P = cand[c];
+                if (tot[c] * p.Hkv >= want) break;
+            }
+        }
+        s_P = P;
+        s_carry = 0;
+    }
+    __syncthreads();
+    const int P = s_P;
+    if (P == 0) {  // plan does not fit: no work, combine writes zero rows
+        for (int b = tid; b < p.batch; b += PLAN_THREADS) p.seq_info[b] = make_int2(0, 0);
+        if (tid == 0) {
+            p.hdr[HDR_N_ITEMS] = 0;
+            p.hdr[HDR_N_UNITS] = 0;
+            p.hdr[HDR_P] = 0;
+            p.hdr[HDR_COUNTER] = 3 * p.total_warps;
+            atomicOr(p.status, PA_STATUS_WORKSPACE | (s_bad ? PA_STATUS_BAD_SEQ_LEN : 0));
+        }
+        return;
+    }
+
+    // ---- pass 2: exclusive scan of partitions per sequence, histogram of item sizes ----
+    const int full_bin = P / BS;
+    for (int base = 0; base < p.batch; base += PLAN_THREADS) {
+        const int b = base + tid;
+        int np = 0;
+        if (b < p.batch) {
+            bool dummy = false;
+            const int L = clamp_len(p.seq_lens[b], max_tok, dummy);
+            np = (L + P - 1) / P;
+            if (np > 0) {
+                if (np > 1) atomicAdd(&hist[full_bin], np - 1);
+                const int last = L - (np - 1) * P;
+                atomicAdd(&hist[(last + BS - 1) / BS], 1);
+            }
+        }
+        int incl = np;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) scan_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int v = scan_warp[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v += u;
+            }
+            scan_warp[lane] = v;  // inclusive over warps
+        }
+        __syncthreads();
+        const int warp_off = warp == 0 ? 0 : scan_warp[warp - 1];
+        const int carry = s_carry;
+        if (b < p.batch) p.seq_info[b] = make_int2(carry + warp_off + incl - np, np);
+        __syncthreads();
+        if (tid == 0) s_carry = carry + scan_warp[31];
+        __syncthreads();
+    }
+    const int n_items = s_carry;
+    if (tid == 0) {
+        int acc = 0;  // larger items first
+        for (int nb = MAX_PART / BS; nb >= 1; --nb) {
+            start[nb] = acc;
+            acc += hist[nb];
+        }
+        p.hdr[HDR_N_ITEMS] = n_items;
+        p.hdr[HDR_N_UNITS] = n_items * p.Hkv;
+        p.hdr[HDR_P] = P;
+        p.hdr[HDR_COUNTER] = 3 * p.total_warps;
+        if (s_bad) atomicOr(p.status, PA_STATUS_BAD_SEQ_LEN);
+    }
+    __syncthreads();
+
+    // ---- pass 3: one warp per sequence, lanes over its partitions ------------------------
+    for (int b = warp; b < p.batch; b += PLAN_THREADS / 32) {
+        bool dummy = false;
+        const int L = clamp_len(p.seq_lens[b], max_tok, dummy);
+        const int np = (L + P - 1) / P;
+        if (np == 0) continue;
+        const int first = p.seq_info[b].x;
+        for (int part = lane; part < np; part += 32) {
+            const int tok0 = part * P;
+            const int ntok = min(P, L - tok0);
+            const int nb = (ntok + BS - 1) / BS;
+            const int pos = start[nb] + atomicAdd(&cursor[nb], 1);
+            p.records[pos] = make_int4(b, tok0, ntok | (np == 1 ? REC_DIRECT : 0), first + part);
+        }
+    }
+}
+
+// ======================================================================================
+// partition attention
+// ======================================================================================
+struct DecodeParams {
+    const __nv_bfloat16* q;
+    __nv_bfloat16* out;
+    const int32_t* block_tables;
+    const int4* records;
+    int* hdr;
+    float* partial_o;    // [item][H][D]  un-normalised
+    float2* partial_ml;  // [item][H]     (running max in log2 units, row sum)
+    int* status;
+    int max_blocks, H, Hkv, G, NB;
+    float scale_log2;
+};
+
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+
+template <int D, bool HI>
+struct UnitRegs {
+    int b, tok0, ntok, pidx, kvh;
+    int nblk;
+    bool direct, valid, bad;
+    int id;                                  // this lane's block id (block index = lane)
+    uint32_t qa[D / 16][HI ? 4 : 2];         // A fragments of Q for every k-step
+};
+
+template <int D, bool HI, int NW, int NSLOT>
+__global__ void __launch_bounds__(NW * 32, 1)
+pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
+                 const __grid_constant__ CUtensorMap vmap, const DecodeParams p) {
+    constexpr int HALVES = D / 64;         // 128-byte swizzled column groups per row
+    constexpr int HALF_BYTES = BS * 128;   // 2 KiB: 16 tokens x 64 dims
+    constexpr int TILE = HALVES * HALF_BYTES;
+    constexpr int SLOT = 2 * TILE;         // K tile then V tile
+    constexpr int KS = D / 16;
+    constexpr int NT = D / 8;
+    constexpr int QW = HI ? 4 : 2;
+    using Unit = UnitRegs<D, HI>;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t slots = base + warp * (NSLOT * SLOT);
+    const uint32_t bars = base + NW * NSLOT * SLOT + warp * (NSLOT * 8);
+
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < NSLOT; ++s) mbar_init(bars + 8 * s, 1);
+        mbar_init_fence();
+        tma_prefetch_desc(&kmap);
+        tma_prefetch_desc(&vmap);
+    }
+    __syncwarp();
+
+    const int n_units = p.hdr[HDR_N_UNITS];
+    const int total_warps = NW * gridDim.x;
+    const int gw = warp * gridDim.x + blockIdx.x;
+    const int G = p.G, H = p.H, Hkv = p.Hkv;
+    const uint32_t* q32 = reinterpret_cast<const uint32_t*>(p.q);
+
+    // ---- unit fetch pipeline: work id -> record -> (block ids, Q fragments) ------------
+    auto load_record = [&](int w, int4& rec, int& kvh, bool& valid) {
+        valid = w < n_units;
+        rec = make_int4(0, 0, 0, 0);
+        kvh = 0;
+        if (valid) {
+            const int item = w / Hkv;
+            kvh = w - item * Hkv;
+            rec = __ldg(&p.records[item]);
+        }
+    };
+    auto build = [&](const int4& rec, int kvh, bool valid, Unit& u) {
+        u.valid = valid;
+        u.b = rec.x;
+        u.tok0 = rec.y;
+        u.ntok = rec.z & 0xFFFF;
+        u.direct = (rec.z & REC_DIRECT) != 0;
+        u.pidx = rec.w;
+        u.kvh = kvh;
+        u.nblk = (u.ntok + BS - 1) / BS;
+        u.bad = false;
+        u.id = 0;
+        if (valid) {
+            if (lane < u.nblk)
+                u.id = __ldg(&p.block_tables[(size_t)u.b * p.max_blocks + u.tok0 / BS + lane]);
+            const size_t row0 = ((size_t)u.b * H + (size_t)kvh * G) * D;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                // a0: (row g, k 2t..), a2: (row g, k 8+2t..); a1/a3 the same for row g+8
+                const size_t c = ks * 16 + 2 * t;
+                u.qa[ks][0] = g < G ? __ldg(&q32[(row0 + (size_t)g * D + c) >> 1]) : 0u;
+                u.qa[ks][QW == 4 ? 2 : 1] =
+                    g < G ? __ldg(&q32[(row0 + (size_t)g * D + c + 8) >> 1]) : 0u;
+                if (HI) {
+                    u.qa[ks][1] = g + 8 < G ? __ldg(&q32[(row0 + (size_t)(g + 8) * D + c) >> 1]) : 0u;
+                    u.qa[ks][QW - 1] =
+                        g + 8 < G ? __ldg(&q32[(row0 + (size_t)(g + 8) * D + c + 8) >> 1]) : 0u;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+                for (int i = 0; i < QW; ++i) u.qa[ks][i] = 0u;
+        }
+    };
+
+    Unit U0, U1;
+    int4 recB;
+    int kvhB;
+    bool validB;
+    int wraw = 0;  // lane 0: work id of the unit after recB
+    {
+        int4 r0, r1;
+        int k0, k1;
+        bool v0, v1;
+        load_record(gw, r0, k0, v0);
+        load_record(gw + total_warps, r1, k1, v1);
+        load_record(gw + 2 * total_warps, recB, kvhB, validB);
+        if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
+        build(r0, k0, v0, U0);
+        build(r1, k1, v1, U1);
+    }
+
+    // ---- per-lane constants of the fragment addresses -------------------------------------
+    // K (B operand, not transposed): matrix i = lane>>3 -> tokens (i>>1)*8.., 16-byte chunk
+    // 2*ks + (i&1); V (B operand, transposed): tokens (i&1)*8.., chunk 2*jj + (i>>1).
+    const int mi = lane >> 3, mr = lane & 7;
+    const uint32_t k_row = ((mi >> 1) * 8 + mr) * 128;
+    const uint32_t k_cb = mi & 1;
+    const uint32_t v_row = ((mi & 1) * 8 + mr) * 128;
+    const uint32_t v_cb = mi >> 1;
+
+    float o[NT][4];
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+
+    uint32_t n_issued = 0, n_done = 0;
+    int iu = 0, ib = 0, cb = 0;  // issue cursor (unit 0/1, block), compute cursor
+    const float sl2 = p.scale_log2;
+
+    while (U0.valid) {
+        // ---- keep the ring full: blocks of U0, then of U1 ---------------------------------
+        while (n_issued - n_done < (uint32_t)NSLOT) {
+            if (iu == 0 && ib == U0.nblk) iu = 1, ib = 0;
+            if (iu == 1 && (!U1.valid || ib == U1.nblk)) break;
+            const int id = __shfl_sync(0xffffffffu, iu ? U1.id : U0.id, ib);
+            const int kvh = iu ? U1.kvh : U0.kvh;
+            if ((unsigned)id >= (unsigned)p.NB) {
+                if (iu) U1.bad = true; else U0.bad = true;
+            }
+            if (lane == 0) {
+                const uint32_t s = n_issued % NSLOT;
+                const uint32_t bar = bars + 8 * s;
+                const uint32_t dst = slots + s * SLOT;
+                mbar_arrive_expect_tx(bar, SLOT);
+                // an id outside the pool is out of the tensor's bounds: TMA fills zeros
+#pragma unroll
+                for (int hf = 0; hf < HALVES; ++hf) {
+                    tma_load_4d(dst + hf * HALF_BYTES, &kmap, bar, hf * 64, 0, kvh, id);
+                    tma_load_4d(dst + TILE + hf * HALF_BYTES, &vmap, bar, hf * 64, 0, kvh, id);
+                }
+            }
+            ++n_issued;
+            ++ib;
+        }
+
+        // ---- one block of U0 -----------------------------------------------------------------
+        {
+            const uint32_t s = n_done % NSLOT;
+            if (!mbar_wait_bounded(bars + 8 * s, (n_done / NSLOT) & 1, WAIT_LIMIT_NS)) {
+                if (lane == 0) atomicOr(p.status, PA_STATUS_TIMEOUT);
+                // give the copies still in flight a bounded chance to land, then leave
+                for (uint32_t c = n_done + 1; c < n_issued; ++c)
+                    mbar_wait_bounded(bars + 8 * (c % NSLOT), (c / NSLOT) & 1, WAIT_LIMIT_NS);
+                return;
+            }
+            const uint32_t kbase = slots + s * SLOT, vbase = kbase + TILE;
+            const int nvalid = min(BS, U0.ntok - cb * BS);
+
+            if (nvalid < BS) {
+                // unused slots of a sequence's last block may hold anything: zero their V rows
+                // (0 * NaN would poison the accumulators); their scores are masked below
+                const int nchunk = (BS - nvalid) * 8;
+                for (int hf = 0; hf < HALVES; ++hf)
+                    for (int c = lane; c < nchunk; c += 32)
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(
+                                         vbase + hf * HALF_BYTES + nvalid * 128 + c * 16),
+                                     "r"(0u)
+                                     : "memory");
+                fence_proxy_async_smem();
+                __syncwarp();
+            }
+
+            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t b00, b01, b10, b11;
+                const uint32_t chunk = ((ks & 3) * 2 + k_cb) ^ mr;
+                ldmatrix_x4(kbase + (ks >> 2) * HALF_BYTES + k_row + (chunk << 4), b00, b01, b10,
+                            b11);
+                const uint32_t a0 = U0.qa[ks][0], a2 = U0.qa[ks][QW == 4 ? 2 : 1];
+                const uint32_t a1 = HI ? U0.qa[ks][1] : 0u, a3 = HI ? U0.qa[ks][QW - 1] : 0u;
+                mma_bf16_16816(s0, a0, a1, a2, a3, b00, b01);
+                mma_bf16_16816(s1, a0, a1, a2, a3, b10, b11);
+            }
+
+            // scale to log2 units, mask tokens past the sequence end
+            const int c0 = 2 * t;
+            const bool v00 = c0 < nvalid, v01 = c0 + 1 < nvalid, v10 = c0 + 8 < nvalid,
+                       v11 = c0 + 9 < nvalid;
+            s0[0] = v00 ? s0[0] * sl2 : -INFINITY;
+            s0[1] = v01 ? s0[1] * sl2 : -INFINITY;
+            s1[0] = v10 ? s1[0] * sl2 : -INFINITY;
+            s1[1] = v11 ? s1[1] * sl2 : -INFINITY;
+            float mx0 = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            const float mn0 = fmaxf(m0, mx0);
+            const float mu0 = mn0 == -INFINITY ? 0.f : mn0;
+            const float corr0 = ex2(m0 - mu0);
+            m0 = mn0;
+            const uint32_t pa0 = pack_bf16x2(ex2(s0[0] - mu0), ex2(s0[1] - mu0));
+            const uint32_t pa2 = pack_bf16x2(ex2(s1[0] - mu0), ex2(s1[1] - mu0));
+            // the row sum uses the rounded weights, the same ones the MMA multiplies by
+            l0 = l0 * corr0 + ((bf16lo_to_f32(pa0) + bf16hi_to_f32(pa0)) +
+                               (bf16lo_to_f32(pa2) + bf16hi_to_f32(pa2)));
+            uint32_t pa1 = 0u, pa3 = 0u;
+            float corr1 = 1.f;
+            if (HI) {
+                s0[2] = v00 ? s0[2] * sl2 : -INFINITY;
+                s0[3] = v01 ? s0[3] * sl2 : -INFINITY;
+                s1[2] = v10 ? s1[2] * sl2 : -INFINITY;
+                s1[3] = v11 ? s1[3] * sl2 : -INFINITY;
+                float mx1 = fmaxf(fmaxf(s0[2], s0[3]), fmaxf(s1[2], s1[3]));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                const float mn1 = fmaxf(m1, mx1);
+                const float mu1 = mn1 == -INFINITY ? 0.f : mn1;
+                corr1 = ex2(m1 - mu1);
+                m1 = mn1;
+                pa1 = pack_bf16x2(ex2(s0[2] - mu1), ex2(s0[3] - mu1));
+                pa3 = pack_bf16x2(ex2(s1[2] - mu1), ex2(s1[3] - mu1));
+                l1 = l1 * corr1 + ((bf16lo_to_f32(pa1) + bf16hi_to_f32(pa1)) +
+                                   (bf16lo_to_f32(pa3) + bf16hi_to_f32(pa3)));
+            }
+            // rescale only when some row's maximum moved (warp-uniform branch)
+            if (__any_sync(0xffffffffu, corr0 != 1.f || corr1 != 1.f)) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    o[nt][0] *= corr0;
+                    o[nt][1] *= corr0;
+                    if (HI) {
+                        o[nt][2] *= corr1;
+                        o[nt][3] *= corr1;
+                    }
+                }
+            }
+
+            // O += P V: V^T fragments straight from the [token][dim] tile
+#pragma unroll
+            for (int jj = 0; jj < D / 16; ++jj) {
+                uint32_t v0, v1, v2, v3;
+                const uint32_t chunk = ((jj & 3) * 2 + v_cb) ^ mr;
+                ldmatrix_x4_trans(vbase + (jj >> 2) * HALF_BYTES + v_row + (chunk << 4), v0, v1,
+                                  v2, v3);
+                mma_bf16_16816(o[2 * jj], pa0, pa1, pa2, pa3, v0, v1);
+                mma_bf16_16816(o[2 * jj + 1], pa0, pa1, pa2, pa3, v2, v3);
+            }
+            ++n_done;
+            ++cb;
+        }
+
+        // ---- unit finished: write its result, move to the next unit -----------------------------
+        if (cb == U0.nblk) {
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+            if (HI) {
+                l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+            }
+            const int h0 = U0.kvh * G + g;
+            if (U0.direct) {
+                const float i0 = U0.bad ? 0.f : 1.f / l0, i1 = U0.bad ? 0.f : 1.f / l1;
+                if (g < G) {
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(p.out + ((size_t)U0.b * H + h0) * D);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0);
+                }
+                if (HI && g + 8 < G) {
+                    uint32_t* dst =
+                        reinterpret_cast<uint32_t*>(p.out + ((size_t)U0.b * H + h0 + 8) * D);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][2] * i1, o[nt][3] * i1);
+                }
+            } else {
+                const float nanv = __int_as_float(0x7fc00000);
+                if (g < G) {
+                    const size_t row = (size_t)U0.pidx * H + h0;
+                    float2* dst = reinterpret_cast<float2*>(p.partial_o + row * D);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) dst[nt * 4 + t] = make_float2(o[nt][0], o[nt][1]);
+                    if (t == 0) p.partial_ml[row] = make_float2(U0.bad ? nanv : m0, l0);
+                }
+                if (HI && g + 8 < G) {
+                    const size_t row = (size_t)U0.pidx * H + h0 + 8;
+                    float2* dst = reinterpret_cast<float2*>(p.partial_o + row * D);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) dst[nt * 4 + t] = make_float2(o[nt][2], o[nt][3]);
+                    if (t == 0) p.partial_ml[row] = make_float2(U0.bad ? nanv : m1, l1);
+                }
+            }
+            // advance the fetch pipeline
+            U0 = U1;
+            build(recB, kvhB, validB, U1);
+            const int w = __shfl_sync(0xffffffffu, wraw, 0);
+            load_record(w, recB, kvhB, validB);
+            if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
+            if (iu == 1) iu = 0; else ib = 0;  // the issue cursor stays where it was
+            cb = 0;
+            m0 = m1 = -INFINITY;
+            l0 = l1 = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+        }
+    }
+}
+
+// ======================================================================================
+// combine: one warp per (sequence, query head)
+// ======================================================================================
+struct CombineParams {
+    const int2* seq_info;
+    const float* partial_o;
+    const float2* partial_ml;
+    __nv_bfloat16* out;
+    int* hdr;
+    int rows;  // batch * H
+    int H;
+    int counter_reset;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) {
+    constexpr int VPL = D / 32;  // floats per lane
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
+    if (row >= p.rows) return;
+    const int b = row / p.H, h = row - b * p.H;
+    const int2 info = p.seq_info[b];
+    if (info.y == 1) return;  // written directly by the attention kernel
+    __nv_bfloat16* dst = p.out + (size_t)row * D + lane * VPL;
+    float acc[VPL];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
+    float den = 0.f;
+    bool bad = false;
+    if (info.y > 1) {
+        float M = -INFINITY;
+        for (int i = lane; i < info.y; i += 32) {
+            const float m = p.partial_ml[(size_t)(info.x + i) * p.H + h].x;
+            bad |= m != m;
+            M = fmaxf(M, m);
+        }
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        bad = __any_sync(0xffffffffu, bad);
+        if (M == -INFINITY) M = 0.f;
+#pragma unroll 4
+        for (int i = 0; i < info.y; ++i) {
+            const size_t r = (size_t)(info.x + i) * p.H + h;
+            const float2 ml = p.partial_ml[r];
+            const float w = ex2(ml.x - M);
+            den += w * ml.y;
+            const float* src = p.partial_o + r * D + lane * VPL;
+            if (VPL == 4) {
+                const float4 v = *reinterpret_cast<const float4*>(src);
+                acc[0] += w * v.x, acc[1] += w * v.y, acc[2] += w * v.z, acc[3] += w * v.w;
+            } else {
+                const float2 v = *reinterpret_cast<const float2*>(src);
+                acc[0] += w * v.x, acc[1] += w * v.y;
+            }
+        }
+    }
+    const float inv = (info.y > 1 && !bad) ? 1.f / den : 0.f;
+    if (VPL == 4) {
+        uint2 v;
+        v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+        v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+        if (inv == 0.f) v.x = v.y = 0u;
+        *reinterpret_cast<uint2*>(dst) = v;
+    } else {
+        uint32_t v = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+        if (inv == 0.f) v = 0u;
+        *reinterpret_cast<uint32_t*>(dst) = v;
+    }
+}
+
+// ======================================================================================
+// host side
+// ======================================================================================
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
+                cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+// tensor map over one layer's cache: dims (dim, slot, kv head, block), box 64 x 16 x 1 x 1
+static int make_cache_map(CUtensorMap* map, const void* base, const pa_shape* s) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) {
+        set_cuda_error((int)cudaErrorSymbolNotFound);
+        return PA_ERR_CUDA;
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)s->head_dim, (cuuint64_t)s->block_size,
+                          (cuuint64_t)s->num_kv_heads, (cuuint64_t)s->num_blocks};
+    cuuint64_t strides[3] = {(cuuint64_t)s->stride_tok * 2, (cuuint64_t)s->stride_head * 2,
+                             (cuuint64_t)s->stride_block * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)BS, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error((int)r);
+        return PA_ERR_CUDA;
+    }
+    return PA_OK;
+}
+
+WsLayout ws_layout(int H, int D, int64_t batch, int64_t item_cap, size_t bytes) {
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    WsLayout w;
+    w.off_seqinfo = up(HDR_WORDS * sizeof(int));
+    w.off_records = w.off_seqinfo + up((size_t)batch * sizeof(int2));
+    const size_t per_item = sizeof(int4) + (size_t)H * sizeof(float2) + (size_t)H * D * sizeof(float);
+    if (bytes > 0) {
+        const size_t fixed = w.off_records + 3 * 256;
+        item_cap = bytes > fixed ? (int64_t)((bytes - fixed) / per_item) : 0;
+    }
+    w.item_cap = item_cap;
+    w.off_ml = w.off_records + up((size_t)item_cap * sizeof(int4));
+    w.off_o = w.off_ml + up((size_t)item_cap * H * sizeof(float2));
+    w.total = w.off_o + up((size_t)item_cap * H * D * sizeof(float));
+    return w;
+}
+
+struct Variant {
+    int nw, nslot;
+};
+
+template <int D, bool HI, int NW, int NSLOT>
+static int launch_decode(const CUtensorMap& km, const CUtensorMap& vm, const DecodeParams& dp,
+                         const DeviceInfo& dev, int* grid_out, bool launch, cudaStream_t st) {
+    auto kern = pa_decode_kernel<D, HI, NW, NSLOT>;
+    const int smem = NW * NSLOT * (2 * BS * D * 2) + NW * NSLOT * 8 + 1024;
+    if (smem > dev.smem_optin) return PA_ERR_SHAPE;
+    static int configured_dev = -1, ctas_per_sm = 0;
+    static std::mutex mu;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (configured_dev != dev.device) {
+            int rc = check_cuda(cudaFuncSetAttribute(
+                kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            if (rc) return rc;
+            rc = check_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas_per_sm, kern,
+                                                                          NW * 32, smem));
+            if (rc) return rc;
+            if (ctas_per_sm < 1) return PA_ERR_SHAPE;
+            configured_dev = dev.device;
+        }
+    }
+    const int grid = dev.sm_count * ctas_per_sm;
+    *grid_out = grid * NW;  // total warps
+    if (!launch) return PA_OK;
+    kern<<<grid, NW * 32, smem, st>>>(km, vm, dp);
+    count_launch();
+    return check_cuda(cudaGetLastError());
+}
+
+template <int D, bool HI>
+static int dispatch_variant(Variant v, const CUtensorMap& km, const CUtensorMap& vm,
+                            const DecodeParams& dp, const DeviceInfo& dev, int* warps, bool launch,
+                            cudaStream_t st) {
+    constexpr int F = 128 / D;  // a D=64 slot is half the size: twice the slots
+#define PK_CASE(NW_, NS_) \
+    if (v.nw == NW_ && v.nslot == NS_) \
+        return launch_decode<D, HI, NW_, NS_ * F>(km, vm, dp, dev, warps, launch, st);
+    PK_CASE(8, 3)
+    PK_CASE(12, 2)
+    PK_CASE(6, 4)
+    PK_CASE(4, 6)
+    PK_CASE(4, 3)
+    PK_CASE(4, 2)
+#undef PK_CASE
+    return PA_ERR_ARG;
+}
+
+static Variant chosen_variant() {
+    static Variant v = [] {
+        Variant d{8, 3};
+        if (const char* e = std::getenv("PAGEDKV_VARIANT")) {
+            int a = 0, b = 0;
+            if (std::sscanf(e, "%d,%d", &a, &b) == 2) d = Variant{a, b};
+        }
+        return d;
+    }();
+    return v;
+}
+
+static int dispatch_decode(const pa_shape* s, const CUtensorMap& km, const CUtensorMap& vm,
+                           const DecodeParams& dp, const DeviceInfo& dev, int* warps, bool launch,
+                           cudaStream_t st) {
+    const bool hi = s->num_q_heads / s->num_kv_heads > 8;
+    const Variant v = chosen_variant();
+    if (s->head_dim == 128)
+        return hi ? dispatch_variant<128, true>(v, km, vm, dp, dev, warps, launch, st)
+                  : dispatch_variant<128, false>(v, km, vm, dp, dev, warps, launch, st);
+    return hi ? dispatch_variant<64, true>(v, km, vm, dp, dev, warps, launch, st)
+              : dispatch_variant<64, false>(v, km, vm, dp, dev, warps, launch, st);
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace pk
+
+using namespace pk;
+
+extern "C" int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch,
+                                  int64_t max_total_tokens, int32_t partition_tokens,
+                                  size_t* bytes) {
+    if (!shape || !bytes) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (max_batch < 0 || max_total_tokens < 0) return PA_ERR_ARG;
+    if (partition_tokens != 0 &&
+        (partition_tokens < BS || partition_tokens > MAX_PART || partition_tokens % BS))
+        return PA_ERR_ARG;
+    const int64_t pw = partition_tokens ? partition_tokens : 256;
+    const int64_t cap = max_total_tokens / pw + max_batch + 1;
+    WsLayout w = ws_layout(shape->num_q_heads, shape->head_dim, max_batch, cap, 0);
+    *bytes = w.total + 3 * 256;
+    return PA_OK;
+}
+
+extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cache,
+                         const void* v_cache, const int32_t* block_tables,
+                         int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
+                         float scale, void* out, void* workspace, size_t workspace_bytes,
+                         int32_t partition_tokens, int32_t flags, int32_t* dev_status,
+                         void* cuda_stream) {
+    if (!shape) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (batch < 0 || max_blocks_per_seq < 0) return PA_ERR_ARG;
+    if (partition_tokens != 0 &&
+        (partition_tokens < BS || partition_tokens > MAX_PART || partition_tokens % BS))
+        return PA_ERR_ARG;
+    if (flags & ~PA_FLAG_REUSE_PLAN) return PA_ERR_ARG;
+    if (batch == 0) return PA_OK;
+    if (!q || !k_cache || !v_cache || !block_tables || !seq_lens || !out || !workspace)
+        return PA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return PA_ERR_ALIGN;
+    if ((int64_t)max_blocks_per_seq * BS > INT32_MAX) return PA_ERR_ARG;
+
+    const int H = shape->num_q_heads, D = shape->head_dim;
+    WsLayout w = ws_layout(H, D, batch, 0, workspace_bytes);
+    if (w.item_cap < batch || w.total > workspace_bytes) return PA_ERR_WORKSPACE;
+
+    DeviceInfo dev;
+    rc = get_device_info(&dev);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* hdr = reinterpret_cast<int*>(ws);
+    int* status = dev_status ? dev_status : hdr + HDR_STATUS;
+
+    CUtensorMap km, vm;
+    rc = make_cache_map(&km, k_cache, shape);
+    if (rc) return rc;
+    rc = make_cache_map(&vm, v_cache, shape);
+    if (rc) return rc;
+
+    DecodeParams dp;
+    dp.q = static_cast<const __nv_bfloat16*>(q);
+    dp.out = static_cast<__nv_bfloat16*>(out);
+    dp.block_tables = block_tables;
+    dp.records = reinterpret_cast<const int4*>(ws + w.off_records);
+    dp.hdr = hdr;
+    dp.partial_o = reinterpret_cast<float*>(ws + w.off_o);
+    dp.partial_ml = reinterpret_cast<float2*>(ws + w.off_ml);
+    dp.status = status;
+    dp.max_blocks = max_blocks_per_seq;
+    dp.H = H;
+    dp.Hkv = shape->num_kv_heads;
+    dp.G = H / shape->num_kv_heads;
+    dp.NB = shape->num_blocks;
+    dp.scale_log2 = scale * 1.4426950408889634f;
+
+    int total_warps = 0;
+    rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, false, st);
+    if (rc) return rc;
+
+    if (!(flags & PA_FLAG_REUSE_PLAN)) {
+        PlanParams pp;
+        pp.seq_lens = seq_lens;
+        pp.batch = batch;
+        pp.max_blocks = max_blocks_per_seq;
+        pp.Hkv = shape->num_kv_heads;
+        pp.forced_p = partition_tokens;
+        pp.item_cap = w.item_cap;
+        pp.total_warps = total_warps;
+        pp.hdr = hdr;
+        pp.seq_info = reinterpret_cast<int2*>(ws + w.off_seqinfo);
+        pp.records = reinterpret_cast<int4*>(ws + w.off_records);
+        pp.status = status;
+        pa_plan_kernel<<<1, PLAN_THREADS, 0, st>>>(pp);
+        count_launch();
+        rc = check_cuda(cudaGetLastError());
+        if (rc) return rc;
+    }
+
+    rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, true, st);
+    if (rc) return rc;
+
+    CombineParams cp;
+    cp.seq_info = reinterpret_cast<const int2*>(ws + w.off_seqinfo);
+    cp.partial_o = dp.partial_o;
+    cp.partial_ml = dp.partial_ml;
+    cp.out = dp.out;
+    cp.hdr = hdr;
+    cp.rows = batch * H;
+    cp.H = H;
+    cp.counter_reset = 3 * total_warps;
+    const int cgrid = (cp.rows + 3) / 4;
+    if (D == 128)
+        pa_combine_kernel<128><<<cgrid, 128, 0, st>>>(cp);
+    else
+        pa_combine_kernel<64><<<cgrid, 128, 0, st>>>(cp);
+    count_launch();
+    return check_cuda(cudaGetLastError());
+}
+
+extern "C" int pa_host_io_bytes(const pa_shape* shape, int32_t max_batch,
+                                int32_t max_blocks_per_seq, size_t* bytes) {
+    if (!shape || !bytes) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (max_batch < 0 || max_blocks_per_seq < 0) return PA_ERR_ARG;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t qo = up((size_t)max_batch * shape->num_q_heads * shape->head_dim * 2);
+    *bytes = 2 * qo + up((size_t)max_batch * max_blocks_per_seq * 4) + up((size_t)max_batch * 4);
+    return PA_OK;
+}
+
+extern "C" int pa_decode_host(const pa_shape* shape, const void* q_host, const void* k_cache,
+                              const void* v_cache, const int32_t* block_tables_host,
+                              int32_t max_blocks_per_seq, const int32_t* seq_lens_host,
+                              int32_t batch, float scale, void* out_host, void* io_buf,
+                              size_t io_bytes, void* workspace, size_t workspace_bytes,
+                              int32_t partition_tokens, int32_t* dev_status, void* cuda_stream) {
+    if (!shape) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (batch < 0 || max_blocks_per_seq < 0) return PA_ERR_ARG;
+    if (batch == 0) return PA_OK;
+    if (!q_host || !block_tables_host || !seq_lens_host || !out_host || !io_buf)
+        return PA_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(io_buf) & 255) return PA_ERR_ALIGN;
+    size_t need = 0;
+    rc = pa_host_io_bytes(shape, batch, max_blocks_per_seq, &need);
+    if (rc) return rc;
+    if (io_bytes < need) return PA_ERR_WORKSPACE;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t qbytes = (size_t)batch * shape->num_q_heads * shape->head_dim * 2;
+    const size_t tbytes = (size_t)batch * max_blocks_per_seq * 4;
+    uint8_t* io = static_cast<uint8_t*>(io_buf);
+    void* dq = io;
+    void* dout = io + up(qbytes);
+    void* dtab = io + 2 * up(qbytes);
+    void* dlen = io + 2 * up(qbytes) + up(tbytes);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    rc = check_cuda(cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = check_cuda(cudaMemcpyAsync(dtab, block_tables_host, tbytes, cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = check_cuda(
+        cudaMemcpyAsync(dlen, seq_lens_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = pa_decode(shape, dq, k_cache, v_cache, static_cast<const int32_t*>(dtab),
+                   max_blocks_per_seq, static_cast<const int32_t*>(dlen), batch, scale, dout,
+                   workspace, workspace_bytes, partition_tokens, 0, dev_status, cuda_stream);
+    if (rc) return rc;
+    return check_cuda(cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, st));
+}
