@@ -176,6 +176,17 @@ int kv_swap_in(const kv_pool_desc* pool, const pa_shape* shape, void* k_pool, vo
                const void* pinned_host_buf, size_t host_bytes, const int32_t* block_ids,
                int32_t n, void* staging, size_t staging_bytes, void* cuda_stream);
 
+/*
+ * Per-kernel timing of pa_decode (no counterpart in the paper; a measurement aid).  While
+ * enabled, every pa_decode call records CUDA events on its stream before the plan kernel,
+ * before and after the partition-attention kernel and after the combine kernel.
+ * pa_profile_read waits for the recorded calls to finish, returns the summed device time of
+ * each kernel in milliseconds and the number of calls, and forgets them.  Any output
+ * pointer may be NULL.  Events are host objects; no device memory is allocated.
+ */
+int pa_profile_enable(int on);
+int pa_profile_read(double* plan_ms, double* attention_ms, double* combine_ms, int64_t* calls);
+
 /* Text for a PA_* return code. */
 const char* pa_status_string(int code);
 

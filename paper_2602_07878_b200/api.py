@@ -28,7 +28,7 @@ ERR = {"NULL": -1, "SHAPE": -2, "ALIGN": -3, "WORKSPACE": -4, "HOSTBUF": -5, "BL
 
 EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
-           "pa_last_cuda_error", "pa_launch_count"]
+           "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read"]
 
 
 class PaShape(ctypes.Structure):
@@ -80,6 +80,11 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = ctypes.c_int
         L.pa_status_string.argtypes = [ctypes.c_int]
         L.pa_status_string.restype = ctypes.c_char_p
+        pd = ctypes.POINTER(ctypes.c_double)
+        L.pa_profile_enable.argtypes = [ctypes.c_int]
+        L.pa_profile_enable.restype = ctypes.c_int
+        L.pa_profile_read.argtypes = [pd, pd, pd, ctypes.POINTER(ctypes.c_int64)]
+        L.pa_profile_read.restype = ctypes.c_int
         L.pa_launch_count.argtypes = []
         L.pa_launch_count.restype = ctypes.c_int64
         _lib = L
@@ -210,3 +215,16 @@ def kv_swap_in(k_pool, v_pool, pinned_host_buf, block_ids, staging=None, stream=
 
 def pa_launch_count() -> int:
     return int(lib().pa_launch_count())
+
+
+def pa_profile_enable(on: bool):
+    _check(lib().pa_profile_enable(1 if on else 0), "pa_profile_enable")
+
+
+def pa_profile_read():
+    """(plan_ms, attention_ms, combine_ms, calls) summed over the calls recorded so far."""
+    t = [ctypes.c_double(0) for _ in range(3)]
+    n = ctypes.c_int64(0)
+    _check(lib().pa_profile_read(ctypes.byref(t[0]), ctypes.byref(t[1]), ctypes.byref(t[2]),
+                                 ctypes.byref(n)), "pa_profile_read")
+    return t[0].value, t[1].value, t[2].value, int(n.value)

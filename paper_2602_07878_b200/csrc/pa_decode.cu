@@ -18,6 +18,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -341,6 +342,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             const int kvh = iu ? U1.kvh : U0.kvh;
             if ((unsigned)id >= (unsigned)p.NB) {
                 if (iu) U1.bad = true; else U0.bad = true;
+                if (lane == 0) atomicOr(p.status, PA_STATUS_BAD_BLOCK_ID);
             }
             if (lane == 0) {
                 const uint32_t s = n_issued % NSLOT;
@@ -729,6 +731,32 @@ static int dispatch_decode(const pa_shape* s, const CUtensorMap& km, const CUten
               : dispatch_variant<64, false>(v, km, vm, dp, dev, warps, launch, st);
 }
 
+// ---- optional per-kernel timing (CUDA events recorded around each of the three launches) ----
+struct ProfCall {
+    cudaEvent_t ev[4];
+};
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<ProfCall> g_prof_calls;
+static std::vector<ProfCall> g_prof_free;
+constexpr size_t PROF_MAX_CALLS = 1 << 16;
+
+static bool prof_begin_call(ProfCall* out) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    if (!g_prof_on || g_prof_calls.size() >= PROF_MAX_CALLS) return false;
+    ProfCall c;
+    if (!g_prof_free.empty()) {
+        c = g_prof_free.back();
+        g_prof_free.pop_back();
+    } else {
+        for (int i = 0; i < 4; ++i)
+            if (cudaEventCreate(&c.ev[i]) != cudaSuccess) return false;
+    }
+    g_prof_calls.push_back(c);
+    *out = c;
+    return true;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 }  // namespace pk
@@ -812,6 +840,9 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, false, st);
     if (rc) return rc;
 
+    ProfCall prof_ev;
+    const bool prof = prof_begin_call(&prof_ev);
+    if (prof) cudaEventRecord(prof_ev.ev[0], st);
     if (!(flags & PA_FLAG_REUSE_PLAN)) {
         PlanParams pp;
         pp.seq_lens = seq_lens;
@@ -831,8 +862,10 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
         if (rc) return rc;
     }
 
+    if (prof) cudaEventRecord(prof_ev.ev[1], st);
     rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, true, st);
     if (rc) return rc;
+    if (prof) cudaEventRecord(prof_ev.ev[2], st);
 
     CombineParams cp;
     cp.seq_info = reinterpret_cast<const int2*>(ws + w.off_seqinfo);
@@ -849,7 +882,39 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     else
         pa_combine_kernel<64><<<cgrid, 128, 0, st>>>(cp);
     count_launch();
-    return check_cuda(cudaGetLastError());
+    rc = check_cuda(cudaGetLastError());
+    if (prof) cudaEventRecord(prof_ev.ev[3], st);
+    return rc;
+}
+
+extern "C" int pa_profile_enable(int on) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = on != 0;
+    return PA_OK;
+}
+
+extern "C" int pa_profile_read(double* plan_ms, double* attention_ms, double* combine_ms,
+                               int64_t* calls) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    double t[3] = {0, 0, 0};
+    int64_t n = 0;
+    int rc = PA_OK;
+    for (ProfCall& c : g_prof_calls) {
+        if (rc == PA_OK) rc = check_cuda(cudaEventSynchronize(c.ev[3]));
+        for (int i = 0; i < 3 && rc == PA_OK; ++i) {
+            float ms = 0.f;
+            rc = check_cuda(cudaEventElapsedTime(&ms, c.ev[i], c.ev[i + 1]));
+            t[i] += ms;
+        }
+        if (rc == PA_OK) ++n;
+        g_prof_free.push_back(c);
+    }
+    g_prof_calls.clear();
+    if (plan_ms) *plan_ms = t[0];
+    if (attention_ms) *attention_ms = t[1];
+    if (combine_ms) *combine_ms = t[2];
+    if (calls) *calls = n;
+    return rc;
 }
 
 extern "C" int pa_host_io_bytes(const pa_shape* shape, int32_t max_batch,

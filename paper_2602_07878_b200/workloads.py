@@ -84,15 +84,36 @@ def hash16_np(idx: np.ndarray, seed: int) -> np.ndarray:
     return (_mix32_np(lo ^ s) & np.uint64(0xFFFF)).astype(np.int64)
 
 
+def _mix32_u32(x: np.ndarray) -> np.ndarray:
+    """murmur-style 32-bit finaliser on a uint32 array, in place (products wrap mod 2^32)."""
+    x ^= x >> np.uint32(16)
+    x *= np.uint32(0x85EBCA6B)
+    x ^= x >> np.uint32(13)
+    x *= np.uint32(0xC2B2AE35)
+    x ^= x >> np.uint32(16)
+    return x
+
+
 def normal_bf16_np(start: int, count: int, seed: int) -> np.ndarray:
-    """bf16 bits (uint16[count]) of stream `seed` at flat indices start .. start+count-1."""
+    """bf16 bits (uint16[count]) of stream `seed` at flat indices start .. start+count-1.
+
+    Same function as `hash16_np` + table lookup, evaluated in uint32 arithmetic on pieces
+    that do not cross a multiple of 2^32 (so the high word is a scalar per piece)."""
     out = np.empty(count, dtype=np.uint16)
     tab = normal_table()
     step = 1 << 22
-    for o in range(0, count, step):
-        n = min(step, count - o)
-        idx = np.arange(start + o, start + o + n, dtype=np.uint64)
-        out[o:o + n] = tab[hash16_np(idx, seed)]
+    o = 0
+    while o < count:
+        s0 = start + o
+        n = min(step, count - o, (1 << 32) - (s0 & 0xFFFFFFFF))
+        hi = s0 >> 32
+        sh = int(_mix32_np(np.array([(hi + (seed & 0xFFFFFFFF)) & 0xFFFFFFFF], np.uint64))[0])
+        x = np.arange(s0 & 0xFFFFFFFF, (s0 & 0xFFFFFFFF) + n, dtype=np.uint64).astype(np.uint32)
+        x ^= np.uint32(sh)
+        _mix32_u32(x)
+        x &= np.uint32(0xFFFF)
+        np.take(tab, x, out=out[o:o + n])
+        o += n
     return out
 
 
@@ -350,15 +371,10 @@ def pools_torch(spec: DecodeSpec, device, layer: int = 0, poison_tails: bool = T
     k = normal_bf16_torch(layer * n, n, spec.seed_k, device).view(shape)
     v = normal_bf16_torch(layer * n, n, spec.seed_v, device).view(shape)
     if poison_tails:
-        nan = torch.tensor(float("nan"), dtype=torch.bfloat16, device=device)
+        k16, v16 = k.view(torch.int16), v.view(torch.int16)
         for blk, slot in tail_slots(spec):
-            k[blk, :, slot:, :] = nan
-            v[blk, :, slot:, :] = nan
-        # keep the host's poison pattern bit for bit
-        kv16 = (k.view(torch.int16), v.view(torch.int16))
-        for blk, slot in tail_slots(spec):
-            for t in kv16:
-                t[blk, :, slot:, :] = np.int16(BF16_NAN_BITS)
+            k16[blk, :, slot:, :] = BF16_NAN_BITS      # same bit pattern as the host pools
+            v16[blk, :, slot:, :] = BF16_NAN_BITS
     return k, v
 
 
