@@ -1,0 +1,507 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-attention decode + KV-swap hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|5] [--impl ours|reference]
+
+One step = one pa_decode call (plan + partition attention + combine) over one synthetic
+batch whose KV cache is resident in HBM.  The headline number is the KV GB/s of that step
+(algorithmic bytes / device time); the swap path (kv_swap_out / kv_swap_in between the
+device pool and pinned host memory) is timed in the same run and reported in the `swap`
+object against the measured host-link rate.  With N > 1 (torchrun) every rank runs the same
+workload on its own GPU (independent replicas, no data-path collective).
+
+Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attention_kv_gbps"
+UNIT = "GB/s"
+
+
+# --------------------------------------------------------------------------------------
+# small helpers
+# --------------------------------------------------------------------------------------
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:  # NVML missing: report no clocks rather than fail the bench
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or getattr(
+            nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(get_reasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                    "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def aggregate_over_ranks(ms_local: float, units_local: float, dist=None):
+    """Whole-job throughput inputs: (max time over ranks, units summed over ranks).
+
+    `dist` is torch.distributed when a process group is initialised, else None.  Works on
+    any backend (NCCL on GPUs, gloo in the CPU test)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms_local, units_local
+    import torch
+
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def sample_sequences(spec, token_budget: int, seed: int = 7):
+    """Seeded random subset of sequences holding about `token_budget` tokens (at least one)."""
+    order = np.random.Generator(np.random.PCG64(seed)).permutation(spec.batch)
+    pick, tot = [], 0
+    for b in order:
+        L = int(spec.seq_lens[b])
+        if pick and tot + L > token_budget:
+            continue
+        pick.append(int(b))
+        tot += L
+        if tot >= token_budget:
+            break
+    return sorted(pick), tot
+
+
+def compact_tables(spec, seqs):
+    """Block ids used by `seqs` (concatenated) and their tables remapped onto 0..n-1."""
+    ids = np.concatenate([spec.blocks_of(b) for b in seqs]).astype(np.int64)
+    remap = {int(p): i for i, p in enumerate(ids)}
+    mb = max(len(spec.blocks_of(b)) for b in seqs)
+    tables = np.zeros((len(seqs), mb), dtype=np.int32)
+    for i, b in enumerate(seqs):
+        blk = spec.blocks_of(b)
+        tables[i, :len(blk)] = [remap[int(p)] for p in blk]
+    return ids, remap, tables, spec.seq_lens[seqs].astype(np.int32)
+
+
+def compact_host_inputs(spec, seqs, q_dev, k_dev, v_dev):
+    """Host copies (bf16 bit patterns) of what the oracle needs for `seqs`: their q rows and
+    their KV blocks gathered into a small pool with remapped tables.  The device tensors were
+    filled by the seeded generator; copying them back reproduces the generator's bits."""
+    import torch
+
+    ids, _, tables, lens = compact_tables(spec, seqs)
+    idx = torch.from_numpy(ids).to(k_dev.device)
+    to_bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    k = to_bits(k_dev[idx])
+    v = to_bits(v_dev[idx])
+    q = to_bits(q_dev[torch.tensor(seqs, device=q_dev.device)])
+    return q, k, v, tables, lens
+
+
+def sample_kv_bytes(spec, lens):
+    return int(lens.astype(np.int64).sum()) * 2 * spec.num_kv_heads * spec.head_dim * 2
+
+
+# --------------------------------------------------------------------------------------
+# swap timing (N = 1 only)
+# --------------------------------------------------------------------------------------
+def bench_swap(args, torch, api, wl, decode_step, decode_bytes):
+    dev = "cuda"
+    layers, hkv, d, nb = 32, 8, 128, args.swap_pool_blocks
+    n_elems = layers * nb * hkv * 16 * d
+    k_pool = wl.normal_bf16_torch(0, n_elems, 0x51, dev).view(layers, nb, hkv, 16, d)
+    v_pool = wl.normal_bf16_torch(0, n_elems, 0x52, dev).view(layers, nb, hkv, 16, d)
+    bb = api.kv_block_bytes(k_pool, v_pool)
+    tokens = [int(t) for t in args.swap_tokens.split(",")]
+    max_blocks = max(tokens) // 16
+    host = torch.empty(max_blocks * bb, dtype=torch.uint8).pin_memory()
+    staging = torch.empty(args.swap_staging_mib << 20, dtype=torch.uint8, device=dev)
+    side = torch.cuda.Stream()
+    rng = np.random.Generator(np.random.PCG64(0x5A))
+
+    def timed(fn, reps=3):
+        best = None
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(side):
+                e0.record(side)
+                fn()
+                e1.record(side)
+            e1.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        return best
+
+    # host-link ceiling: one contiguous pinned copy (up to 2 GiB) per direction
+    link_bytes = min(max_blocks * bb, 2 << 30)
+    dev_buf = torch.empty(link_bytes, dtype=torch.uint8, device=dev)
+    d2h = timed(lambda: host[:link_bytes].copy_(dev_buf, non_blocking=True))
+    h2d = timed(lambda: dev_buf.copy_(host[:link_bytes], non_blocking=True))
+    link = {"bytes": link_bytes, "d2h_gbps": link_bytes / d2h / 1e6,
+            "h2d_gbps": link_bytes / h2d / 1e6}
+    del dev_buf
+
+    rows = []
+    for n_tok in tokens:
+        n = n_tok // 16
+        perm = rng.permutation(nb)
+        src, dst = perm[:n].astype(np.int32), perm[n:2 * n].astype(np.int32)
+        nbytes = n * bb
+        row = {"tokens": n_tok, "blocks": n, "bytes": nbytes}
+        for mode, stg in (("staged", staging), ("direct", None)):
+            t_out = timed(lambda: api.kv_swap_out(k_pool, v_pool, src, host, stg, stream=side))
+            t_in = timed(lambda: api.kv_swap_in(k_pool, v_pool, host, dst, stg, stream=side))
+            row[mode] = {"out_gbps": nbytes / t_out / 1e6, "in_gbps": nbytes / t_in / 1e6,
+                         "out_frac_of_link": nbytes / t_out / 1e6 / link["d2h_gbps"],
+                         "in_frac_of_link": nbytes / t_in / 1e6 / link["h2d_gbps"]}
+        rows.append(row)
+
+    # churn: evict + restore on the side stream while decode steps run on the main stream
+    n = tokens[-1] // 16
+    perm = rng.permutation(nb)
+    src, dst = perm[:n].astype(np.int32), perm[n:2 * n].astype(np.int32)
+    nbytes = n * bb
+
+    def churn_once():
+        api.kv_swap_out(k_pool, v_pool, src, host, staging, stream=side)
+        api.kv_swap_in(k_pool, v_pool, host, dst, staging, stream=side)
+
+    t_alone = timed(churn_once, reps=1)
+    main = torch.cuda.current_stream()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        e[0].record(side)
+        churn_once()
+        e[1].record(side)
+    steps = 0
+    e[2].record(main)
+    t_host0 = time.perf_counter()
+    while not e[1].query() and time.perf_counter() - t_host0 < 5.0:
+        for _ in range(8):
+            decode_step()
+        steps += 8
+        e[3].record(main)
+        e[3].synchronize()
+    torch.cuda.synchronize()
+    churn = {"tokens": tokens[-1], "swap_bytes_each_way": nbytes,
+             "swap_alone_gbps": 2 * nbytes / t_alone / 1e6,
+             "swap_overlapped_gbps": 2 * nbytes / e[0].elapsed_time(e[1]) / 1e6,
+             "decode_overlapped_gbps": steps * decode_bytes / e[2].elapsed_time(e[3]) / 1e6,
+             "decode_steps_during_swap": steps}
+    return {"pool": {"layers": layers, "kv_heads": hkv, "head_dim": d, "blocks": nb,
+                     "block_bytes": bb, "staging_mib": args.swap_staging_mib},
+            "host_link": link, "sizes": rows, "churn": churn}
+
+
+# --------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+
+    from paper_2602_07878_b200 import api, build as lib_build
+    from paper_2602_07878_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        lib_build.build()
+    if dist is not None:
+        dist.barrier()
+    dev = "cuda"
+
+    spec = wl.config_spec(args.workload)
+    q = wl.q_torch(spec, dev)
+    k, v = wl.pools_torch(spec, dev)
+    tables = torch.from_numpy(spec.block_tables).to(dev)
+    lens = torch.from_numpy(spec.seq_lens).to(dev)
+    out = torch.empty_like(q)
+    shape = api.shape_of(k, spec.num_q_heads)
+    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, spec.total_tokens + 16 * spec.batch),
+                     dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    step_bytes = spec.algorithmic_bytes()
+
+    def step():
+        api.pa_decode(q, k, v, tables, lens, spec.scale, out, ws, dev_status=status)
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+
+    # ---- timed region: exactly K steps between two events on the launching stream ------
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = api.pa_launch_count()
+    api.pa_profile_read()
+    api.pa_profile_enable(True)
+    with ClockSampler(local) as clocks:
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+    api.pa_profile_enable(False)
+    plan_ms, attn_ms, comb_ms, calls = api.pa_profile_read()
+    launches = api.pa_launch_count() - n0
+    ms_local = e0.elapsed_time(e1)
+    if dist is not None:
+        dist.barrier()
+    ms, total_bytes = aggregate_over_ranks(ms_local, float(step_bytes) * args.steps, dist)
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    value = total_bytes / ms / 1e6                      # GB/s over all ranks
+    hdr = ws[:256].view(torch.int32).cpu().numpy()
+
+    # ---- end to end: per-step inputs from pinned host memory, result read back ----------
+    qh, th, lh = q.cpu().pin_memory(), tables.cpu().pin_memory(), lens.cpu().pin_memory()
+    oh = torch.empty_like(qh).pin_memory()
+    io = torch.empty(api.pa_host_io_bytes(shape, spec.batch, th.shape[1]), dtype=torch.uint8,
+                     device=dev)
+
+    def step_e2e():
+        api.pa_decode_host(qh, k, v, th, lh, spec.scale, oh, io, ws, dev_status=status)
+
+    for _ in range(3):
+        step_e2e()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_e2e, bytes_e2e = aggregate_over_ranks(e0.elapsed_time(e1), float(step_bytes) * args.steps,
+                                             dist)
+    assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+    h2d = qh.numel() * 2 + th.numel() * 4 + lh.numel() * 4
+    d2h = oh.numel() * 2
+
+    peak, peak_src = measured_peaks()
+    attn_avg_ms = attn_ms / max(calls, 1)
+    achieved = step_bytes / attn_avg_ms / 1e6
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "num_q_heads": spec.num_q_heads,
+                   "num_kv_heads": spec.num_kv_heads, "head_dim": spec.head_dim,
+                   "block_size": spec.block_size, "pool_blocks": spec.num_blocks,
+                   "total_context_tokens": spec.total_tokens,
+                   "kv_bytes_per_step": spec.kv_bytes(), "algorithmic_bytes_per_step": step_bytes,
+                   "partition_tokens": int(hdr[2]), "work_items": int(hdr[0]),
+                   "l2": "inputs (KV read per step) exceed the 126 MB L2; no flush",
+                   "parallelism": "independent replicas" if world > 1 else "1 gpu"},
+        "tokens_per_s": world * spec.batch * args.steps / (ms / 1e3),
+        "frac_of_hbm_peak": value / world / peak,
+        "frac_of_nominal_8tbs": value / world / 8000.0,
+        "e2e": {"value": bytes_e2e / ms_e2e / 1e6, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "kernels_ms_per_step": {"plan": plan_ms / max(calls, 1), "attention": attn_avg_ms,
+                                "combine": comb_ms / max(calls, 1)},
+        "roofline": {"bound": "hbm", "kernel": "pa_decode_kernel", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": NCU_TRAFFIC.get(spec.name), "peak_source": peak_src},
+        "clocks": clocks.summary(),
+    }
+
+    if rank == 0 and world == 1:
+        if not args.no_swap:
+            line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
+        if not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline(args, spec, q, k, v)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one pa_decode_kernel launch, from the ncu
+# capture summarised under profiles/ (None until a capture of the current kernel exists)
+NCU_TRAFFIC = {}
+
+
+def cpu_baseline(args, spec, q, k, v):
+    """The fp64 oracle, as it stands, on the host cores, over a bounded sample of the batch."""
+    import oracle
+
+    budget = int(spec.total_tokens * args.cpu_fraction)
+    seqs, tot = sample_sequences(spec, budget)
+    qh, kh, vh, tables, lens = compact_host_inputs(spec, seqs, q, k, v)
+    t0 = time.perf_counter()
+    oracle.pa_decode(qh, kh, vh, tables, lens, spec.scale)
+    dt = time.perf_counter() - t0
+    return {"value": sample_kv_bytes(spec, lens) / dt / 1e9, "unit": UNIT,
+            "cores": oracle.threads(), "kind": "oracle", "seconds": dt,
+            "sample": f"{len(seqs)} of {spec.batch} sequences of {spec.name} "
+                      f"({tot} of {spec.total_tokens} context tokens), one pass"}
+
+
+# --------------------------------------------------------------------------------------
+# reference arm: the oracle on the host cores
+# --------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2602_07878_b200 import workloads as wl
+
+    spec = wl.config_spec(args.workload)
+    # size the per-step sample so that warmup + steps end within a couple of minutes:
+    # the oracle streams roughly 0.2 GB/s of KV per core
+    est_gbps = 0.2 * oracle.threads()
+    budget_bytes = 120.0 / max(1, args.steps + args.warmup) * est_gbps * 1e9
+    tok_bytes = 2 * spec.num_kv_heads * spec.head_dim * 2
+    budget_tok = int(min(spec.total_tokens, max(256, budget_bytes / tok_bytes)))
+    seqs, tot = sample_sequences(spec, budget_tok)
+    try:
+        import torch
+
+        have_gpu = torch.cuda.is_available()
+    except Exception:
+        have_gpu = False
+    if have_gpu:
+        # generator output produced on the device and copied back (same bits as on the host)
+        q = wl.q_torch(spec, "cuda")
+        k, v = wl.pools_torch(spec, "cuda")
+        qh, kh, vh, tables, lens = compact_host_inputs(spec, seqs, q, k, v)
+        del q, k, v
+    else:
+        ids, remap, tables, lens = compact_tables(spec, seqs)
+        kh, vh = wl.pool_block_np(spec, "k", ids), wl.pool_block_np(spec, "v", ids)
+        for blk, slot in wl.tail_slots(spec):
+            if blk in remap:
+                kh[remap[blk], :, slot:] = wl.BF16_NAN_BITS
+                vh[remap[blk], :, slot:] = wl.BF16_NAN_BITS
+        qh = wl.q_np(spec)[seqs]
+    nbytes = sample_kv_bytes(spec, lens)
+    for _ in range(args.warmup):
+        oracle.pa_decode(qh, kh, vh, tables, lens, spec.scale)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.pa_decode(qh, kh, vh, tables, lens, spec.scale)
+    dt = time.perf_counter() - t0
+    value = nbytes * args.steps / dt / 1e9
+    sample = (f"{len(seqs)} of {spec.batch} sequences of {spec.name} ({tot} of "
+              f"{spec.total_tokens} context tokens) per step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "num_q_heads": spec.num_q_heads,
+                   "num_kv_heads": spec.num_kv_heads, "head_dim": spec.head_dim,
+                   "block_size": spec.block_size, "pool_blocks": spec.num_blocks,
+                   "total_context_tokens": spec.total_tokens},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 5],
+                    help="decode workload (3 = full-pool mixed-length GQA, the headline)")
+    ap.add_argument("--no-swap", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-fraction", type=float, default=1.0,
+                    help="fraction of the batch's tokens the CPU baseline pass covers")
+    ap.add_argument("--swap-pool-blocks", type=int, default=6144)
+    ap.add_argument("--swap-tokens", default="1024,4096,16384")
+    ap.add_argument("--swap-staging-mib", type=int, default=256)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
