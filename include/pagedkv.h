@@ -41,6 +41,7 @@ extern "C" {
 #define PA_ERR_BLOCK_ID (-6)  /* swap block id out of range or listed twice                */
 #define PA_ERR_CUDA (-7)      /* a CUDA runtime/driver call failed; see pa_last_cuda_error */
 #define PA_ERR_ARG (-8)       /* negative count, bad partition size or similar             */
+#define PA_ERR_STATIC_LIMIT (-9) /* pa_decode_static: needs more than PA_STATIC_WORKSPACE_BYTES */
 
 /* ---- bits OR-ed into *dev_status by the kernels -------------------------------------- */
 #define PA_STATUS_BAD_SEQ_LEN 1   /* seq_lens[b] < 0 or > max_blocks_per_seq * block_size  */
@@ -122,6 +123,44 @@ int pa_decode(const pa_shape* shape, const void* q, const void* k_cache, const v
               const int32_t* block_tables, int32_t max_blocks_per_seq, const int32_t* seq_lens,
               int32_t batch, float scale, void* out, void* workspace, size_t workspace_bytes,
               int32_t partition_tokens, int32_t flags, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * pa_decode for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this is a convenience of the library.)
+ *
+ * Some users of this library are never in a position to call cudaMalloc for the workspace
+ * pa_decode wants: an attention backend loaded into a serving engine that handed the whole
+ * GPU to its KV pool at start-up and forbids later allocation, a plug-in that is only given
+ * the tensors of the current step, or a latency-critical loop that must not hit the implicit
+ * device synchronisation of the allocator.  For them the library carries its own scratch: a
+ * fixed array of PA_STATIC_WORKSPACE_BYTES in device memory that belongs to the loaded
+ * module.  Every GPU on which the library is loaded gives up that much memory until the
+ * process exits, whether or not this entry point is ever called.
+ *
+ * Arguments are those of pa_decode without workspace / workspace_bytes / flags, plus
+ *   max_total_tokens   an upper bound on the sum of seq_lens (the host cannot read them).
+ * The call computes pa_workspace_bytes(shape, batch, max_total_tokens, partition_tokens)
+ * and returns PA_ERR_STATIC_LIMIT, launching nothing, if that exceeds
+ * PA_STATIC_WORKSPACE_BYTES.  (If the bound was understated the plan may not fit; that is
+ * reported through PA_STATUS_WORKSPACE like in pa_decode and the output rows are zero.)
+ * It calls no cudaMalloc / cudaFree and no allocating library routine; inputs and outputs
+ * are still the caller's.
+ *
+ * First call on each device: the array's device address is looked up once per device (with
+ * that device current) and cached.  Make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array, and it keeps what the last call left
+ * there.  The call clears the plan header before use; everything else is overwritten
+ * before it is read.  Two calls whose GPU work overlaps (different streams, or different
+ * host threads feeding different streams) race on the array and corrupt each other's
+ * results: serialise them on one stream or with events.  Plan reuse is not offered here for
+ * the same reason.
+ */
+#define PA_STATIC_WORKSPACE_BYTES (64u << 20)
+int pa_decode_static(const pa_shape* shape, const void* q, const void* k_cache,
+                     const void* v_cache, const int32_t* block_tables,
+                     int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
+                     int64_t max_total_tokens, float scale, void* out, int32_t partition_tokens,
+                     int32_t* dev_status, void* cuda_stream);
 
 /* Bytes of device buffer pa_decode_host needs for its device copies of q, block tables,
  * lengths and out. */

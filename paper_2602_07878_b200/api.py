@@ -24,11 +24,13 @@ PA_STATUS_BAD_BLOCK_ID = 2
 PA_STATUS_TIMEOUT = 4
 PA_STATUS_WORKSPACE = 8
 ERR = {"NULL": -1, "SHAPE": -2, "ALIGN": -3, "WORKSPACE": -4, "HOSTBUF": -5, "BLOCK_ID": -6,
-       "CUDA": -7, "ARG": -8}
+       "CUDA": -7, "ARG": -8, "STATIC_LIMIT": -9}
+PA_STATIC_WORKSPACE_BYTES = 64 << 20
 
 EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
-           "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read"]
+           "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
+           "pa_decode_static"]
 
 
 class PaShape(ctypes.Structure):
@@ -69,6 +71,9 @@ def lib() -> ctypes.CDLL:
         L.pa_workspace_bytes.argtypes = [pshape, i32, i64, i32, psz]
         L.pa_decode.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp, sz,
                                 i32, i32, vp, vp]
+        L.pa_decode_static.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, i64, ctypes.c_float,
+                                       vp, i32, vp, vp]
+        L.pa_decode_static.restype = ctypes.c_int
         L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
         L.pa_decode_host.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp,
                                      sz, vp, sz, i32, vp, vp]
@@ -228,3 +233,20 @@ def pa_profile_read():
     _check(lib().pa_profile_read(ctypes.byref(t[0]), ctypes.byref(t[1]), ctypes.byref(t[2]),
                                  ctypes.byref(n)), "pa_profile_read")
     return t[0].value, t[1].value, t[2].value, int(n.value)
+
+
+def pa_decode_static(q, k_cache, v_cache, block_tables, seq_lens, scale, out, max_total_tokens, *,
+                     partition_tokens: int = 0, dev_status=None, stream=None):
+    """Forward to pa_decode_static: pa_decode without a caller workspace.  The scratch is a
+    fixed array inside the library (PA_STATIC_WORKSPACE_BYTES per GPU), shared by all calls,
+    so calls must not overlap on the GPU; `max_total_tokens` bounds the sum of seq_lens."""
+    shape = shape_of(k_cache, q.shape[1])
+    assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
+    assert block_tables.dtype == torch.int32 and seq_lens.dtype == torch.int32
+    assert q.is_contiguous() and out.is_contiguous() and block_tables.is_contiguous()
+    rc = lib().pa_decode_static(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                _ptr(block_tables), block_tables.shape[1], _ptr(seq_lens),
+                                q.shape[0], int(max_total_tokens), float(scale), _ptr(out),
+                                partition_tokens, _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_decode_static")
+    return out

@@ -71,6 +71,8 @@ extern "C" const char* pa_status_string(int code) {
         case PA_ERR_BLOCK_ID: return "block id out of range or duplicated";
         case PA_ERR_CUDA: return "CUDA call failed (see pa_last_cuda_error)";
         case PA_ERR_ARG: return "invalid argument";
+        case PA_ERR_STATIC_LIMIT:
+            return "request needs more scratch than the built-in static workspace holds";
         default: return "unknown status";
     }
 }

@@ -969,3 +969,54 @@ extern "C" int pa_decode_host(const pa_shape* shape, const void* q_host, const v
     if (rc) return rc;
     return check_cuda(cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, st));
 }
+
+// ======================================================================================
+// pa_decode_static: the same three kernels, scratch taken from a fixed device array
+// ======================================================================================
+// The array below is part of the loaded module: every GPU that loads this library sets
+// PA_STATIC_WORKSPACE_BYTES aside for it until the process exits.  In host code the name
+// `g_static_workspace` is only a handle for the runtime; the device address that kernels
+// can use comes from cudaGetSymbolAddress, asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_workspace[PA_STATIC_WORKSPACE_BYTES];
+
+static int static_workspace_address(void** out) {
+    static std::mutex mu;
+    static void* addr[64] = {nullptr};
+    int dev = 0;
+    int rc = pk::check_cuda(cudaGetDevice(&dev));
+    if (rc) return rc;
+    if (dev < 0 || dev >= 64) return PA_ERR_ARG;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        rc = pk::check_cuda(cudaGetSymbolAddress(&p, g_static_workspace));
+        if (rc) return rc;
+        if (!p) return PA_ERR_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return PA_OK;
+}
+
+extern "C" int pa_decode_static(const pa_shape* shape, const void* q, const void* k_cache,
+                                const void* v_cache, const int32_t* block_tables,
+                                int32_t max_blocks_per_seq, const int32_t* seq_lens,
+                                int32_t batch, int64_t max_total_tokens, float scale, void* out,
+                                int32_t partition_tokens, int32_t* dev_status,
+                                void* cuda_stream) {
+    size_t need = 0;
+    int rc = pa_workspace_bytes(shape, batch, max_total_tokens, partition_tokens, &need);
+    if (rc) return rc;
+    if (need > (size_t)PA_STATIC_WORKSPACE_BYTES) return PA_ERR_STATIC_LIMIT;
+    if (batch == 0) return PA_OK;
+    void* ws = nullptr;
+    rc = static_workspace_address(&ws);
+    if (rc) return rc;
+    // the array still holds the previous call's plan header and fallback status word
+    rc = pk::check_cuda(cudaMemsetAsync(ws, 0, pk::HDR_WORDS * sizeof(int),
+                                        static_cast<cudaStream_t>(cuda_stream)));
+    if (rc) return rc;
+    return pa_decode(shape, q, k_cache, v_cache, block_tables, max_blocks_per_seq, seq_lens, batch,
+                     scale, out, ws, (size_t)PA_STATIC_WORKSPACE_BYTES, partition_tokens, 0,
+                     dev_status, cuda_stream);
+}
