@@ -177,7 +177,7 @@ def bench_swap(args, torch, api, wl, decode_step, decode_bytes):
     bb = api.kv_block_bytes(k_pool, v_pool)
     tokens = [int(t) for t in args.swap_tokens.split(",")]
     max_blocks = max(tokens) // 16
-    host = torch.empty(max_blocks * bb, dtype=torch.uint8).pin_memory()
+    host = torch.empty(max_blocks * bb, dtype=torch.uint8, pin_memory=True)
     staging = torch.empty(args.swap_staging_mib << 20, dtype=torch.uint8, device=dev)
     side = torch.cuda.Stream()
     rng = np.random.Generator(np.random.PCG64(0x5A))

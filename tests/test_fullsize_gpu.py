@@ -1,0 +1,162 @@
+"""Parity at the full workload sizes, in the launch configuration bench.py times
+(automatic partition size, device-generated inputs): sampled sequences are recomputed by the
+fp64 oracle from inputs regenerated on the CPU; properties that hold for every row are
+checked on all rows."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_07878_b200 import api
+from paper_2602_07878_b200 import workloads as wl
+from helpers import assert_parity, torch_to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def host_inputs_for(spec, seqs, layer=0):
+    """q rows, compact K/V pools and remapped tables of `seqs`, regenerated with numpy."""
+    ids = np.concatenate([spec.blocks_of(b) for b in seqs]).astype(np.int64)
+    remap = {int(p): i for i, p in enumerate(ids)}
+    k = wl.pool_block_np(spec, "k", ids, layer)
+    v = wl.pool_block_np(spec, "v", ids, layer)
+    if layer == 0:
+        for blk, slot in wl.tail_slots(spec):
+            if blk in remap:
+                k[remap[blk], :, slot:] = wl.BF16_NAN_BITS
+                v[remap[blk], :, slot:] = wl.BF16_NAN_BITS
+    mb = max(len(spec.blocks_of(b)) for b in seqs)
+    tables = np.zeros((len(seqs), mb), np.int32)
+    for i, b in enumerate(seqs):
+        blk = spec.blocks_of(b)
+        tables[i, :len(blk)] = [remap[int(p)] for p in blk]
+    H, D = spec.num_q_heads, spec.head_dim
+    q = np.stack([wl.normal_bf16_np(b * H * D, H * D, spec.seed_q).reshape(H, D) for b in seqs])
+    return q, k, v, tables, spec.seq_lens[seqs].astype(np.int32), ids
+
+
+def pick(spec, n_long, n_other, seed=3):
+    rng = np.random.default_rng(seed)
+    order = np.argsort(-spec.seq_lens.astype(np.int64), kind="stable")
+    longs = [int(b) for b in order[:n_long]]
+    rest = [int(b) for b in rng.permutation(order[n_long:])[:n_other]]
+    shortest = int(order[-1])
+    return sorted(set(longs + rest + [shortest]))
+
+
+def decode_full(spec, k, v, q=None):
+    dev = "cuda"
+    q = wl.q_torch(spec, dev) if q is None else q
+    tables = torch.from_numpy(spec.block_tables).to(dev)
+    lens = torch.from_numpy(spec.seq_lens).to(dev)
+    out = torch.full_like(q, float("nan"))
+    shape = api.shape_of(k, spec.num_q_heads)
+    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, spec.total_tokens + 16 * spec.batch),
+                     dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    api.pa_decode(q, k, v, tables, lens, spec.scale, out, ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    hdr = ws[:256].view(torch.int32).cpu().numpy()
+    return q, out, hdr
+
+
+@pytest.mark.parametrize("index,n_long,n_other", [(2, 2, 6), (3, 1, 12), (5, 1, 2)])
+def test_full_size_decode_sampled_against_oracle(index, n_long, n_other):
+    spec = wl.config_spec(index)
+    k, v = wl.pools_torch(spec, "cuda")
+    q, out, hdr = decode_full(spec, k, v)
+    # every row: finite, and a convex mixture of N(0,1)-table values cannot leave their range
+    assert torch.isfinite(out).all()
+    assert float(out.float().abs().max()) <= 4.25
+    assert int(hdr[0]) >= spec.batch and int(hdr[2]) in (64, 128, 256, 512)
+    seqs = pick(spec, n_long, n_other)
+    qh, kh, vh, tables, lens, ids = host_inputs_for(spec, seqs)
+    # the device generator and the host generator give the same bits
+    some = ids[:: max(1, len(ids) // 16)]
+    dev_bits = k[torch.from_numpy(some).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
+    assert (dev_bits == kh[:: max(1, len(ids) // 16)]).all()
+    assert (q[seqs].view(torch.int16).cpu().numpy().view(np.uint16) == qh).all()
+    ref = oracle.pa_decode(qh, kh, vh, tables, lens, spec.scale)
+    assert_parity(torch_to_f64(out[seqs]), ref, spec.name)
+
+
+def test_full_size_swap_churn_and_decode():
+    """Workload 4 at full size: 32-layer pool of 60000 blocks at 98 % occupancy; evict 64K
+    tokens' worth of whole sequences, restore them into other blocks, decode one layer."""
+    free, total = torch.cuda.mem_get_info()
+    if free < 150 * (1 << 30):
+        pytest.skip("needs about 140 GB of free device memory")
+    spec = wl.config_spec(4)
+    dev = "cuda"
+    layers, nb = spec.num_layers, spec.num_blocks
+    n = nb * spec.block_elems
+    shape5 = (layers, nb, spec.num_kv_heads, 16, spec.head_dim)
+    k_pool = wl.normal_bf16_torch(0, layers * n, spec.seed_k, dev).view(shape5)
+    v_pool = wl.normal_bf16_torch(0, layers * n, spec.seed_v, dev).view(shape5)
+    seqs, src, dst = wl.pick_victims(spec, 65536, seed=11)
+    assert len(src) == 4096 and len(set(dst.tolist())) == 4096
+    bb = api.kv_block_bytes(k_pool, v_pool)
+    assert bb == 2 << 20
+    host = torch.empty(len(src) * bb, dtype=torch.uint8, pin_memory=True)
+    staging = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def checksum(exclude):
+        keep = torch.ones(nb, dtype=torch.bool, device=dev)
+        keep[torch.from_numpy(np.asarray(exclude, dtype=np.int64)).to(dev)] = False
+        tot = 0
+        for pool in (k_pool, v_pool):
+            for l in range(layers):
+                x = pool[l].view(torch.int16).view(nb, -1)
+                tot += int((x.sum(dim=1, dtype=torch.int64) * keep).sum().item())
+        return tot
+
+    before = checksum(dst)
+    api.kv_swap_out(k_pool, v_pool, src, host, staging)
+    torch.cuda.synchronize()
+    img = host.numpy().view(np.uint16).reshape(len(src), layers, 2, -1)
+    rng = np.random.default_rng(0)
+    for i in rng.integers(0, len(src), 6):
+        for layer in (0, 13, 31):
+            assert (img[i, layer, 0] == wl.pool_block_np(spec, "k", [src[i]], layer).reshape(-1)).all()
+            assert (img[i, layer, 1] == wl.pool_block_np(spec, "v", [src[i]], layer).reshape(-1)).all()
+    src_t = torch.from_numpy(src.astype(np.int64)).to(dev)
+    dst_t = torch.from_numpy(dst.astype(np.int64)).to(dev)
+    # the freed blocks get overwritten before the victims come back (unless reused as targets)
+    reused = set(dst.tolist())
+    trash = torch.from_numpy(np.array([p for p in src if p not in reused], dtype=np.int64)).to(dev)
+    expect_k = k_pool[:, src_t].clone()
+    expect_v = v_pool[:, src_t].clone()
+    trash_sum = sum(int(p[:, trash].view(torch.int16).sum(dtype=torch.int64).item())
+                    for p in (k_pool, v_pool))
+    k_pool[:, trash] = float("nan")
+    v_pool[:, trash] = float("nan")
+    api.kv_swap_in(k_pool, v_pool, host, dst, None)          # direct mode on the way back
+    torch.cuda.synchronize()
+    assert torch.equal(k_pool[:, dst_t].view(torch.int16), expect_k.view(torch.int16))
+    assert torch.equal(v_pool[:, dst_t].view(torch.int16), expect_v.view(torch.int16))
+    del expect_k, expect_v
+    # bytes outside the destination blocks did not change (the trashed ones are zeroed and
+    # their original content, summed on the device beforehand, is subtracted)
+    k_pool[:, trash] = 0
+    v_pool[:, trash] = 0
+    after = checksum(dst)
+    before_adj = before - trash_sum
+    assert after == before_adj
+
+    # decode layer 7 over the whole batch with the victims remapped to their new blocks
+    layer = 7
+    t = spec.block_tables.copy()
+    o = 0
+    for b in seqs:
+        nblk = min(len(spec.blocks_of(b)), len(dst) - o)
+        t[b, :nblk] = dst[o:o + nblk]
+        o += nblk
+    spec2 = wl.DecodeSpec(**{**spec.__dict__, "block_tables": t})
+    q, out, hdr = decode_full(spec2, k_pool[layer], v_pool[layer])
+    assert torch.isfinite(out).all()
+    sample = sorted(set(pick(spec, 1, 4) + seqs[:2]))
+    # oracle inputs from the CPU generator at the ORIGINAL block ids (content moved with the swap)
+    qh, kh, vh, tables, lens, ids = host_inputs_for(spec, sample, layer)
+    ref = oracle.pa_decode(qh, kh, vh, tables, lens, spec.scale)
+    assert_parity(torch_to_f64(out[sample]), ref, "workload 4 decode after churn")
