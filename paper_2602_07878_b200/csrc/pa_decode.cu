@@ -525,7 +525,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
 }
 
 // ======================================================================================
-// combine: one warp per (sequence, query head)
+// combine: one CTA per (sequence, query head)
 // ======================================================================================
 struct CombineParams {
     const int2* seq_info;
@@ -538,59 +538,87 @@ struct CombineParams {
     int counter_reset;
 };
 
+// One CTA (4 warps) per (sequence, query head) row.  Every warp finds the row maximum, then
+// the warps share the partitions (warp w takes w, w+4, ...), eight independent 512-byte row
+// loads at a time, and the four partial sums meet in shared memory.
 template <int D>
 __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) {
     constexpr int VPL = D / 32;  // floats per lane
-    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (blockIdx.x == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
-    if (row >= p.rows) return;
+    constexpr int UB = 8;        // rows in flight per warp
+    __shared__ float s_acc[4][D];
+    __shared__ float s_den[4];
+    const int row = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (row == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
     const int b = row / p.H, h = row - b * p.H;
     const int2 info = p.seq_info[b];
     if (info.y == 1) return;  // written directly by the attention kernel
-    __nv_bfloat16* dst = p.out + (size_t)row * D + lane * VPL;
+    __nv_bfloat16* dst = p.out + (size_t)row * D;
+    if (info.y == 0) {  // no tokens: a row of zeros
+        if (threadIdx.x < D / 2) reinterpret_cast<uint32_t*>(dst)[threadIdx.x] = 0u;
+        return;
+    }
+    const int np = info.y, first = info.x;
+    float M = -INFINITY;
+    bool bad = false;
+    for (int i = lane; i < np; i += 32) {
+        const float m = p.partial_ml[(size_t)(first + i) * p.H + h].x;
+        bad |= m != m;  // NaN marks a partition that met a bad block id
+        M = fmaxf(M, m);
+    }
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    bad = __any_sync(0xffffffffu, bad);
+    if (M == -INFINITY) M = 0.f;
+
     float acc[VPL];
 #pragma unroll
     for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
     float den = 0.f;
-    bool bad = false;
-    if (info.y > 1) {
-        float M = -INFINITY;
-        for (int i = lane; i < info.y; i += 32) {
-            const float m = p.partial_ml[(size_t)(info.x + i) * p.H + h].x;
-            bad |= m != m;
-            M = fmaxf(M, m);
-        }
-        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-        bad = __any_sync(0xffffffffu, bad);
-        if (M == -INFINITY) M = 0.f;
-#pragma unroll 4
-        for (int i = 0; i < info.y; ++i) {
-            const size_t r = (size_t)(info.x + i) * p.H + h;
-            const float2 ml = p.partial_ml[r];
-            const float w = ex2(ml.x - M);
-            den += w * ml.y;
+    for (int i0 = warp; i0 < np; i0 += 4 * UB) {
+        float2 ml[UB];
+        float v[UB][VPL];
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            const size_t r = (size_t)(first + min(i0 + 4 * u, np - 1)) * p.H + h;
+            ml[u] = p.partial_ml[r];
             const float* src = p.partial_o + r * D + lane * VPL;
             if (VPL == 4) {
-                const float4 v = *reinterpret_cast<const float4*>(src);
-                acc[0] += w * v.x, acc[1] += w * v.y, acc[2] += w * v.z, acc[3] += w * v.w;
+                const float4 x = *reinterpret_cast<const float4*>(src);
+                v[u][0] = x.x, v[u][1] = x.y, v[u][VPL - 2] = x.z, v[u][VPL - 1] = x.w;
             } else {
-                const float2 v = *reinterpret_cast<const float2*>(src);
-                acc[0] += w * v.x, acc[1] += w * v.y;
+                const float2 x = *reinterpret_cast<const float2*>(src);
+                v[u][0] = x.x, v[u][1] = x.y;
             }
         }
+#pragma unroll
+        for (int u = 0; u < UB; ++u)
+            if (i0 + 4 * u < np) {
+                const float w = ex2(ml[u].x - M);
+                den += w * ml[u].y;
+#pragma unroll
+                for (int i = 0; i < VPL; ++i) acc[i] += w * v[u][i];
+            }
     }
-    const float inv = (info.y > 1 && !bad) ? 1.f / den : 0.f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) s_acc[warp][lane * VPL + i] = acc[i];
+    if (lane == 0) s_den[warp] = den;
+    __syncthreads();
+    if (warp != 0) return;
+    den = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
+    const float inv = bad ? 0.f : 1.f / den;
+    float o[VPL];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+        const int c = lane * VPL + i;
+        o[i] = ((s_acc[0][c] + s_acc[1][c]) + (s_acc[2][c] + s_acc[3][c])) * inv;
+    }
     if (VPL == 4) {
-        uint2 v;
-        v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-        v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-        if (inv == 0.f) v.x = v.y = 0u;
-        *reinterpret_cast<uint2*>(dst) = v;
+        uint2 x;
+        x.x = bad ? 0u : pack_bf16x2(o[0], o[1]);
+        x.y = bad ? 0u : pack_bf16x2(o[VPL - 2], o[VPL - 1]);
+        *reinterpret_cast<uint2*>(dst + lane * VPL) = x;
     } else {
-        uint32_t v = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-        if (inv == 0.f) v = 0u;
-        *reinterpret_cast<uint32_t*>(dst) = v;
+        *reinterpret_cast<uint32_t*>(dst + lane * VPL) = bad ? 0u : pack_bf16x2(o[0], o[1]);
     }
 }
 
@@ -698,11 +726,7 @@ static int dispatch_variant(Variant v, const CUtensorMap& km, const CUtensorMap&
     if (v.nw == NW_ && v.nslot == NS_) \
         return launch_decode<D, HI, NW_, NS_ * F>(km, vm, dp, dev, warps, launch, st);
     PK_CASE(8, 3)
-    PK_CASE(12, 2)
-    PK_CASE(6, 4)
-    PK_CASE(4, 6)
     PK_CASE(4, 3)
-    PK_CASE(4, 2)
 #undef PK_CASE
     return PA_ERR_ARG;
 }
@@ -876,7 +900,7 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     cp.rows = batch * H;
     cp.H = H;
     cp.counter_reset = 3 * total_warps;
-    const int cgrid = (cp.rows + 3) / 4;
+    const int cgrid = cp.rows;
     if (D == 128)
         pa_combine_kernel<128><<<cgrid, 128, 0, st>>>(cp);
     else
