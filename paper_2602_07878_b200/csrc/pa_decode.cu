@@ -18,6 +18,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "internal.h"
@@ -62,6 +63,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int max_tok = p.max_blocks * BS;
     const int cand[4] = {64, 128, 256, 512};
+    pdl_launch_dependents();  // the attention kernel may set up while the plan is made
+    pdl_wait();               // the workspace may still be in use by the previous call
 
     // ---- pass 1: item counts for each candidate partition size ------------------------
     long long cnt[5] = {0, 0, 0, 0, 0};
@@ -244,6 +247,8 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         tma_prefetch_desc(&vmap);
     }
     __syncwarp();
+    pdl_launch_dependents();  // combine CTAs may take their seats; they wait for this grid
+    pdl_wait();               // the plan (and everything before it) is complete and visible
 
     const int n_units = p.hdr[HDR_N_UNITS];
     const int total_warps = NW * gridDim.x;
@@ -549,6 +554,8 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) 
     __shared__ float s_den[4];
     const int row = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();  // partial results of the attention kernel are complete and visible
     if (row == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
     const int b = row / p.H, h = row - b * p.H;
     const int2 info = p.seq_info[b];
@@ -684,6 +691,24 @@ WsLayout ws_layout(int H, int D, int64_t batch, int64_t item_cap, size_t bytes) 
     return w;
 }
 
+// Launch with programmatic stream serialization: the kernel may start before the previous
+// kernel in the stream has finished and synchronises on it with griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 struct Variant {
     int nw, nslot;
 };
@@ -712,9 +737,8 @@ static int launch_decode(const CUtensorMap& km, const CUtensorMap& vm, const Dec
     const int grid = dev.sm_count * ctas_per_sm;
     *grid_out = grid * NW;  // total warps
     if (!launch) return PA_OK;
-    kern<<<grid, NW * 32, smem, st>>>(km, vm, dp);
     count_launch();
-    return check_cuda(cudaGetLastError());
+    return check_cuda(launch_pdl(kern, dim3(grid), dim3(NW * 32), smem, st, km, vm, dp));
 }
 
 template <int D, bool HI>
@@ -880,9 +904,8 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
         pp.seq_info = reinterpret_cast<int2*>(ws + w.off_seqinfo);
         pp.records = reinterpret_cast<int4*>(ws + w.off_records);
         pp.status = status;
-        pa_plan_kernel<<<1, PLAN_THREADS, 0, st>>>(pp);
         count_launch();
-        rc = check_cuda(cudaGetLastError());
+        rc = check_cuda(launch_pdl(pa_plan_kernel, dim3(1), dim3(PLAN_THREADS), 0, st, pp));
         if (rc) return rc;
     }
 
@@ -901,12 +924,9 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     cp.H = H;
     cp.counter_reset = 3 * total_warps;
     const int cgrid = cp.rows;
-    if (D == 128)
-        pa_combine_kernel<128><<<cgrid, 128, 0, st>>>(cp);
-    else
-        pa_combine_kernel<64><<<cgrid, 128, 0, st>>>(cp);
     count_launch();
-    rc = check_cuda(cudaGetLastError());
+    rc = check_cuda(D == 128 ? launch_pdl(pa_combine_kernel<128>, dim3(cgrid), dim3(128), 0, st, cp)
+                             : launch_pdl(pa_combine_kernel<64>, dim3(cgrid), dim3(128), 0, st, cp));
     if (prof) cudaEventRecord(prof_ev.ev[3], st);
     return rc;
 }

@@ -17,6 +17,14 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
+// ---- programmatic dependent launch -------------------------------------------------------
+// wait: blocks until the grids this one depends on have finished and their writes are visible.
+// launch_dependents: lets the next grid in the stream start its own prologue early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- mbarrier -------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
