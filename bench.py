@@ -240,12 +240,14 @@ def bench_swap(args, torch, api, wl, decode_step, decode_bytes):
     steps = 0
     e[2].record(main)
     t_host0 = time.perf_counter()
-    while not e[1].query() and time.perf_counter() - t_host0 < 5.0:
+    while True:
         for _ in range(8):
             decode_step()
         steps += 8
         e[3].record(main)
         e[3].synchronize()
+        if e[1].query() or time.perf_counter() - t_host0 > 5.0:
+            break
     torch.cuda.synchronize()
     churn = {"tokens": tokens[-1], "swap_bytes_each_way": nbytes,
              "swap_alone_gbps": 2 * nbytes / t_alone / 1e6,
