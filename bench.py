@@ -358,7 +358,12 @@ def run_ours(args):
     ms_e2e, bytes_e2e = aggregate_over_ranks(e0.elapsed_time(e1), float(step_bytes) * args.steps,
                                              dist)
     assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
-    h2d = qh.numel() * 2 + th.numel() * 4 + lh.numel() * 4
+    # q and lengths are copied; table entries are fetched in place over the link, once per
+    # (work item, KV head); output rows are posted in place
+    used_entries = int(((spec.seq_lens.astype(np.int64) + spec.block_size - 1) // spec.block_size).sum())
+    table_bytes = th.numel() * 4
+    h2d = qh.numel() * 2 + lh.numel() * 4 + (used_entries * 4 * spec.num_kv_heads
+                                             if table_bytes >= (256 << 10) else table_bytes)
     d2h = oh.numel() * 2
 
     peak, peak_src = measured_peaks()

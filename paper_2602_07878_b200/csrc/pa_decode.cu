@@ -1000,17 +1000,38 @@ extern "C" int pa_decode_host(const pa_shape* shape, const void* q_host, const v
     void* dtab = io + 2 * up(qbytes);
     void* dlen = io + 2 * up(qbytes) + up(tbytes);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // Pinned memory the GPU can address is used in place: block-table entries are fetched two
+    // work units ahead of their use, and output rows are posted as they are produced, so both
+    // transfers overlap the kernels instead of preceding / following them.  q is re-read by
+    // every partition of a sequence and is copied once instead.
+    auto mapped = [](const void* host) -> void* {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
+    };
+    // a small table is cheaper to copy than to read entry by entry over the link
+    void* tab_dev = tbytes >= (256u << 10) ? mapped(block_tables_host) : nullptr;
+    void* out_dev = mapped(out_host);
+    if (out_dev && (reinterpret_cast<uintptr_t>(out_dev) & 15)) out_dev = nullptr;
     rc = check_cuda(cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, st));
     if (rc) return rc;
-    rc = check_cuda(cudaMemcpyAsync(dtab, block_tables_host, tbytes, cudaMemcpyHostToDevice, st));
-    if (rc) return rc;
+    if (!tab_dev) {
+        rc = check_cuda(
+            cudaMemcpyAsync(dtab, block_tables_host, tbytes, cudaMemcpyHostToDevice, st));
+        if (rc) return rc;
+        tab_dev = dtab;
+    }
     rc = check_cuda(
         cudaMemcpyAsync(dlen, seq_lens_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st));
     if (rc) return rc;
-    rc = pa_decode(shape, dq, k_cache, v_cache, static_cast<const int32_t*>(dtab),
-                   max_blocks_per_seq, static_cast<const int32_t*>(dlen), batch, scale, dout,
-                   workspace, workspace_bytes, partition_tokens, 0, dev_status, cuda_stream);
-    if (rc) return rc;
+    rc = pa_decode(shape, dq, k_cache, v_cache, static_cast<const int32_t*>(tab_dev),
+                   max_blocks_per_seq, static_cast<const int32_t*>(dlen), batch, scale,
+                   out_dev ? out_dev : dout, workspace, workspace_bytes, partition_tokens, 0,
+                   dev_status, cuda_stream);
+    if (rc || out_dev) return rc;
     return check_cuda(cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, st));
 }
 
