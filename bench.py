@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the paged-attention decode + KV-swap hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|5] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|4|5] [--impl ours|reference]
 
 One step = one pa_decode call (plan + partition attention + combine) over one synthetic
 batch whose KV cache is resident in HBM.  The headline number is the KV GB/s of that step
@@ -493,14 +493,154 @@ def run_reference(args):
     }))
 
 
+# --------------------------------------------------------------------------------------
+# workload 4: preemption swap churn at full size (1 GPU)
+# --------------------------------------------------------------------------------------
+def run_churn(args):
+    """32-layer pool of 60000 blocks at 98 % occupancy.  For each eviction size N the victims'
+    blocks go to pinned host memory and come back into other blocks on a side stream while
+    the remaining batch is decoded, layer by layer, on the main stream.  One decode step =
+    32 pa_decode calls (one per layer; the plan is made once and reused)."""
+    import torch
+
+    from paper_2602_07878_b200 import api, build as lib_build
+    from paper_2602_07878_b200 import workloads as wl
+
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("workload 4 holds 126 GB per GPU and is run on one GPU")
+    lib_build.build()
+    torch.cuda.set_device(0)
+    dev = "cuda"
+    spec = wl.config_spec(4)
+    layers, nb = spec.num_layers, spec.num_blocks
+    n = nb * spec.block_elems
+    shape5 = (layers, nb, spec.num_kv_heads, 16, spec.head_dim)
+    k_pool = wl.normal_bf16_torch(0, layers * n, spec.seed_k, dev).view(shape5)
+    v_pool = wl.normal_bf16_torch(0, layers * n, spec.seed_v, dev).view(shape5)
+    q = wl.q_torch(spec, dev)
+    tables = torch.from_numpy(spec.block_tables).to(dev)
+    out = torch.empty_like(q)
+    shape = api.shape_of(k_pool[0], spec.num_q_heads)
+    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, spec.total_tokens + 16 * spec.batch),
+                     dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    bb = api.kv_block_bytes(k_pool, v_pool)
+    tokens = [1024, 4096, 16384, 65536]
+    host = torch.empty(tokens[-1] // 16 * bb, dtype=torch.uint8, pin_memory=True)
+    staging = torch.empty(args.swap_staging_mib << 20, dtype=torch.uint8, device=dev)
+    side, main = torch.cuda.Stream(), torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    # host-link ceiling
+    link_bytes = 2 << 30
+    dev_buf = torch.empty(link_bytes, dtype=torch.uint8, device=dev)
+    link = {}
+    for name, fn in (("d2h_gbps", lambda: host[:link_bytes].copy_(dev_buf, non_blocking=True)),
+                     ("h2d_gbps", lambda: dev_buf.copy_(host[:link_bytes], non_blocking=True))):
+        best = 0.0
+        for _ in range(3):
+            a, b = ev(), ev()
+            a.record(main); fn(); b.record(main); b.synchronize()
+            best = max(best, link_bytes / a.elapsed_time(b) / 1e6)
+        link[name] = best
+    del dev_buf
+    link_both = 2.0 / (1.0 / link["d2h_gbps"] + 1.0 / link["h2d_gbps"])
+
+    rows = []
+    with ClockSampler(0) as clocks:
+        for n_tok in tokens:
+            seqs, src, dst = wl.pick_victims(spec, n_tok, seed=100 + n_tok)
+            lens_np = spec.seq_lens.copy()
+            lens_np[seqs] = 0                       # the victims are not in the running batch
+            lens = torch.from_numpy(lens_np).to(dev)
+            step_bytes = layers * dataclass_replace(spec, lens_np).algorithmic_bytes()
+
+            def decode_step():
+                for layer in range(layers):
+                    api.pa_decode(q, k_pool[layer], v_pool[layer], tables, lens, spec.scale, out,
+                                  ws, flags=api.PA_FLAG_REUSE_PLAN if layer else 0,
+                                  dev_status=status)
+
+            def swap_round():
+                api.kv_swap_out(k_pool, v_pool, src, host, staging, stream=side)
+                api.kv_swap_in(k_pool, v_pool, host, dst, staging, stream=side)
+                # and back, so that every round starts from the same pool
+                api.kv_swap_out(k_pool, v_pool, dst, host, staging, stream=side)
+                api.kv_swap_in(k_pool, v_pool, host, src, staging, stream=side)
+
+            nbytes = len(src) * bb
+            for _ in range(2):
+                decode_step()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record(main)
+            for _ in range(args.churn_steps):
+                decode_step()
+            b.record(main); b.synchronize()
+            dec_alone = args.churn_steps * step_bytes / a.elapsed_time(b) / 1e6
+            a, b = ev(), ev()
+            with torch.cuda.stream(side):
+                a.record(side); swap_round(); b.record(side)
+            b.synchronize()
+            swap_alone = 4 * nbytes / a.elapsed_time(b) / 1e6
+            # overlapped
+            e = [ev() for _ in range(4)]
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                e[0].record(side); swap_round(); e[1].record(side)
+            steps = 0
+            e[2].record(main)
+            t0 = time.perf_counter()
+            while True:
+                decode_step()
+                steps += 1
+                e[3].record(main); e[3].synchronize()
+                if e[1].query() or time.perf_counter() - t0 > 20.0:
+                    break
+            torch.cuda.synchronize()
+            rows.append({"tokens": n_tok, "blocks": int(len(src)), "bytes_each_way": nbytes,
+                         "victim_sequences": len(seqs),
+                         "swap_alone_gbps": swap_alone,
+                         "swap_alone_frac_of_link": swap_alone / link_both,
+                         "swap_overlapped_gbps": 4 * nbytes / e[0].elapsed_time(e[1]) / 1e6,
+                         "decode_alone_gbps": dec_alone,
+                         "decode_overlapped_gbps": steps * step_bytes / e[2].elapsed_time(e[3]) / 1e6,
+                         "decode_steps_during_swap": steps,
+                         "decode_step_bytes": step_bytes})
+    assert int(status.item()) == 0
+    peak, peak_src = measured_peaks()
+    best = max(r["decode_alone_gbps"] for r in rows)
+    print(json.dumps({
+        "metric": METRIC, "value": best, "unit": UNIT, "n_gpus": 1, "steps": args.churn_steps,
+        "warmup": 2, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "layers": layers,
+                   "pool_blocks": nb, "allocated_blocks": nb - len(spec.free_blocks),
+                   "pool_bytes": 2 * layers * n * 2, "block_bytes": bb,
+                   "total_context_tokens": spec.total_tokens,
+                   "step": "32 pa_decode calls (one per layer, plan reused) over the non-evicted batch",
+                   "staging_mib": args.swap_staging_mib},
+        "frac_of_hbm_peak": best / peak, "peak_source": peak_src,
+        "host_link": dict(link, harmonic_mean_gbps=link_both),
+        "churn": rows, "clocks": clocks.summary()}))
+
+
+def dataclass_replace(spec, seq_lens):
+    import dataclasses
+
+    return dataclasses.replace(spec, seq_lens=seq_lens)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 5],
-                    help="decode workload (3 = full-pool mixed-length GQA, the headline)")
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5],
+                    help="decode workload (3 = full-pool mixed-length GQA, the headline; "
+                         "4 = full-size swap churn, 126 GB pool, 1 GPU)")
+    ap.add_argument("--churn-steps", type=int, default=3)
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-fraction", type=float, default=1.0,
@@ -510,7 +650,11 @@ def main():
     ap.add_argument("--swap-staging-mib", type=int, default=256)
     args = ap.parse_args()
     if args.impl == "reference":
+        if args.workload == 4:
+            args.workload = 3      # the oracle arm times decode attention; 4 shares 3's mix
         run_reference(args)
+    elif args.workload == 4:
+        run_churn(args)
     else:
         run_ours(args)
 
