@@ -41,6 +41,8 @@ def _load():
         lib.oracle_swap_out.restype = ctypes.c_int
         lib.oracle_swap_in.argtypes = swap
         lib.oracle_swap_in.restype = ctypes.c_int
+        lib.oracle_kv_append.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i64, i64, i64]
+        lib.oracle_kv_append.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -114,3 +116,19 @@ def swap_in(k_pool, v_pool, host, block_ids):
                                 sb, sh, st, _ptr(ids), len(ids), _ptr(host))
     if rc != 0:
         raise ValueError("oracle_swap_in: block id out of range")
+
+
+def kv_append(k_cache, v_cache, k_new, v_new, slot_mapping):
+    """Write token b's K/V rows (uint16[B,Hkv,D]) into flat slot slot_mapping[b] of one
+    layer's caches (uint16[NB,Hkv,bs,D], modified in place); negative slots are skipped."""
+    NB, Hkv, bs, D = k_cache.shape
+    sb, sh, st = _elem_strides(k_cache)
+    assert _elem_strides(v_cache) == (sb, sh, st)
+    k_new = np.ascontiguousarray(k_new, dtype=np.uint16)
+    v_new = np.ascontiguousarray(v_new, dtype=np.uint16)
+    slots = np.ascontiguousarray(slot_mapping, dtype=np.int64)
+    assert k_new.shape == (len(slots), Hkv, D) and v_new.shape == k_new.shape
+    rc = _load().oracle_kv_append(_ptr(k_cache), _ptr(v_cache), _ptr(k_new), _ptr(v_new),
+                                  _ptr(slots), len(slots), Hkv, D, bs, NB, sb, sh, st)
+    if rc != 0:
+        raise ValueError("oracle_kv_append: slot beyond the pool")

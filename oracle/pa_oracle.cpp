@@ -22,6 +22,7 @@
 //   come back into newly allocated blocks): a byte copy of whole blocks, all layers,
 //   K then V, into / out of a contiguous host image laid out
 //   [block i][layer][K|V][kv head][slot][dim].
+//   Append (Section 2.2): the new token's K/V rows are written into their slot.
 //
 // Pins (tests, CPU only): brute-force dense attention without max subtraction in long
 // double on un-paged copies, closed forms (L = 1, L = 2 logistic weights, equal keys ->
@@ -170,6 +171,31 @@ int oracle_swap_in(uint16_t* k_pool, uint16_t* v_pool, int32_t num_layers,
                         for (int d = 0; d < D; ++d)
                             pool[p * stride_block + h * stride_head + t * stride_tok + d] =
                                 host[o++];
+            }
+    }
+    return 0;
+}
+
+// KV append (Section 2.2 "KV-Cache": with every decoding step the new token's K and V
+// vectors are appended to the cache).  Token b goes to flat slot slot_mapping[b] =
+// block * bs + offset of one layer's cache; a negative slot means "no token" (padding).
+// Returns -1 (nothing guaranteed written) if a slot is beyond the pool.
+int oracle_kv_append(uint16_t* k_cache, uint16_t* v_cache, const uint16_t* k_new,
+                     const uint16_t* v_new, const int64_t* slot_mapping, int32_t batch,
+                     int32_t Hkv, int32_t D, int32_t bs, int32_t num_blocks, int64_t stride_block,
+                     int64_t stride_head, int64_t stride_tok) {
+    for (int b = 0; b < batch; ++b)
+        if (slot_mapping[b] >= static_cast<int64_t>(num_blocks) * bs) return -1;
+    for (int b = 0; b < batch; ++b) {
+        const int64_t slot = slot_mapping[b];
+        if (slot < 0) continue;
+        const int64_t p = slot / bs, t = slot % bs;
+        for (int h = 0; h < Hkv; ++h)
+            for (int d = 0; d < D; ++d) {
+                const int64_t dst = p * stride_block + h * stride_head + t * stride_tok + d;
+                const int64_t src = (static_cast<int64_t>(b) * Hkv + h) * D + d;
+                k_cache[dst] = k_new[src];
+                v_cache[dst] = v_new[src];
             }
     }
     return 0;
