@@ -396,6 +396,7 @@ def run_ours(args):
     }
 
     if rank == 0 and world == 1:
+        line["kv_append"] = bench_append(torch, api, spec, k, v)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -405,6 +406,34 @@ def run_ours(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def bench_append(torch, api, spec, k, v, calls=200):
+    """kv_append of one token per sequence into its last slot (the rows written are the ones
+    already there, so the pool keeps its content).  Launch-latency bound: reported in us
+    between back-to-back calls issued from Python."""
+    lens = spec.seq_lens.astype(np.int64)
+    rows = np.nonzero(lens > 0)[0]
+    pos = lens[rows] - 1
+    blk = spec.block_tables[rows, pos // spec.block_size].astype(np.int64)
+    slots_np = np.full(spec.batch, -1, np.int64)
+    slots_np[rows] = blk * spec.block_size + pos % spec.block_size
+    slots = torch.from_numpy(slots_np).cuda()
+    safe = slots.clamp(min=0)
+    k_new = k[safe // 16, :, safe % 16, :].contiguous()
+    v_new = v[safe // 16, :, safe % 16, :].contiguous()
+    for _ in range(5):
+        api.kv_append(k, v, k_new, v_new, slots)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(calls):
+        api.kv_append(k, v, k_new, v_new, slots)
+    e1.record()
+    e1.synchronize()
+    nbytes = 2 * 2 * k_new.numel() * 2          # K and V rows, read + written
+    us = e0.elapsed_time(e1) * 1e3 / calls
+    return {"us_per_call": us, "tokens": int(len(rows)), "bytes": nbytes,
+            "gbps": nbytes / us / 1e3, "bound": "launch latency / host issue rate (2 MB moved per call)"}
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pa_decode_kernel launch, from the ncu

@@ -183,6 +183,24 @@ int pa_decode_host(const pa_shape* shape, const void* q_host, const void* k_cach
                    size_t workspace_bytes, int32_t partition_tokens, int32_t* dev_status,
                    void* cuda_stream);
 
+/*
+ * KV append (Section 2.2 "KV-Cache": with every decoding step the KV vectors of the newly
+ * generated token are appended to the cache).  For every b < batch with slot_mapping[b] >= 0
+ * the rows k_new[b,:,:] and v_new[b,:,:] are written to slot (slot_mapping[b] % block_size)
+ * of physical block (slot_mapping[b] / block_size) of one layer's caches.
+ *
+ *   k_cache, v_cache  dev bf16, one layer, laid out per `shape` (written in place)
+ *   k_new, v_new      dev bf16 [batch, Hkv, D], contiguous, 16-byte aligned
+ *   slot_mapping      dev int64 [batch]; negative = padding entry, nothing is written;
+ *                     a slot at or beyond num_blocks * block_size writes nothing and sets
+ *                     PA_STATUS_BAD_BLOCK_ID in *dev_status (dev int32 or NULL)
+ * Two tokens mapped to the same slot in one call leave either one there.  One kernel is
+ * enqueued on `cuda_stream`.
+ */
+int kv_append(const pa_shape* shape, void* k_cache, void* v_cache, const void* k_new,
+              const void* v_new, const int64_t* slot_mapping, int32_t batch,
+              int32_t* dev_status, void* cuda_stream);
+
 /* Bytes of one block's host image: num_layers * 2 * Hkv * block_size * D * 2. */
 int kv_block_bytes(const kv_pool_desc* pool, const pa_shape* shape, size_t* bytes);
 

@@ -30,7 +30,7 @@ PA_STATIC_WORKSPACE_BYTES = 64 << 20
 EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
-           "pa_decode_static"]
+           "pa_decode_static", "kv_append"]
 
 
 class PaShape(ctypes.Structure):
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.pa_decode_static.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, i64, ctypes.c_float,
                                        vp, i32, vp, vp]
         L.pa_decode_static.restype = ctypes.c_int
+        L.kv_append.argtypes = [pshape, vp, vp, vp, vp, vp, i32, vp, vp]
+        L.kv_append.restype = ctypes.c_int
         L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
         L.pa_decode_host.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp,
                                      sz, vp, sz, i32, vp, vp]
@@ -250,3 +252,16 @@ def pa_decode_static(q, k_cache, v_cache, block_tables, seq_lens, scale, out, ma
                                 partition_tokens, _ptr(dev_status), _stream(stream))
     _check(rc, "pa_decode_static")
     return out
+
+
+def kv_append(k_cache, v_cache, k_new, v_new, slot_mapping, *, dev_status=None, stream=None):
+    """Forward to kv_append: write k_new/v_new [B,Hkv,D] into flat slots slot_mapping (int64
+    [B], negative = skip) of one layer's caches [NB,Hkv,bs,D]."""
+    shape = shape_of(k_cache, k_cache.shape[1])
+    assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
+    assert slot_mapping.dtype == torch.int64 and k_new.is_contiguous() and v_new.is_contiguous()
+    assert k_new.dtype == torch.bfloat16 and k_new.shape == v_new.shape
+    rc = lib().kv_append(ctypes.byref(shape), _ptr(k_cache), _ptr(v_cache), _ptr(k_new),
+                         _ptr(v_new), _ptr(slot_mapping), k_new.shape[0], _ptr(dev_status),
+                         _stream(stream))
+    _check(rc, "kv_append")
