@@ -41,6 +41,9 @@ def _load():
         lib.oracle_swap_out.restype = ctypes.c_int
         lib.oracle_swap_in.argtypes = swap
         lib.oracle_swap_in.restype = ctypes.c_int
+        lib.oracle_pa_prefill.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, i32, i32, i32, i32, i32,
+                                          i64, i64, i64, dbl, vp, i32]
+        lib.oracle_pa_prefill.restype = ctypes.c_int
         lib.oracle_kv_append.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i64, i64, i64]
         lib.oracle_kv_append.restype = ctypes.c_int
         _lib = lib
@@ -132,3 +135,27 @@ def kv_append(k_cache, v_cache, k_new, v_new, slot_mapping):
                                   _ptr(slots), len(slots), Hkv, D, bs, NB, sb, sh, st)
     if rc != 0:
         raise ValueError("oracle_kv_append: slot beyond the pool")
+
+
+def pa_prefill(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, num_threads: int = 0):
+    """fp64 causal attention [total_q, H, D] of packed query tokens over the paged cache.
+
+    q uint16[total_q,H,D]; sequence b owns rows cu_q_lens[b]..cu_q_lens[b+1]-1, which are the
+    last tokens of its ctx_lens[b] cached tokens."""
+    q = np.ascontiguousarray(q, dtype=np.uint16)
+    block_tables = np.ascontiguousarray(block_tables, dtype=np.int32)
+    ctx_lens = np.ascontiguousarray(ctx_lens, dtype=np.int32)
+    cu = np.ascontiguousarray(cu_q_lens, dtype=np.int32)
+    T, H, D = q.shape
+    NB, Hkv, bs, _ = k_cache.shape
+    B = len(ctx_lens)
+    assert len(cu) == B + 1 and (B == 0 or cu[-1] == T)
+    sb, sh, st = _elem_strides(k_cache)
+    assert _elem_strides(v_cache) == (sb, sh, st)
+    out = np.zeros((T, H, D), dtype=np.float64)
+    rc = _load().oracle_pa_prefill(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
+                                   block_tables.shape[1], _ptr(ctx_lens), _ptr(cu), B, H, Hkv, D,
+                                   bs, NB, sb, sh, st, float(scale), _ptr(out), num_threads)
+    if rc != 0:
+        raise ValueError("oracle_pa_prefill: inconsistent lengths or bad block id")
+    return out

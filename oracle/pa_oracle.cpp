@@ -23,6 +23,8 @@
 //   K then V, into / out of a contiguous host image laid out
 //   [block i][layer][K|V][kv head][slot][dim].
 //   Append (Section 2.2): the new token's K/V rows are written into their slot.
+//   Prefill (Sections 2.1, 5.1.2 "Recomputation"): causal attention of a chunk of query
+//   tokens over the paged cache, the definition above applied per query position.
 //
 // Pins (tests, CPU only): brute-force dense attention without max subtraction in long
 // double on un-paged copies, closed forms (L = 1, L = 2 logistic weights, equal keys ->
@@ -197,6 +199,78 @@ int oracle_kv_append(uint16_t* k_cache, uint16_t* v_cache, const uint16_t* k_new
                 k_cache[dst] = k_new[src];
                 v_cache[dst] = v_new[src];
             }
+    }
+    return 0;
+}
+
+// Prefill / recomputation attention (Section 2.1 "Prefill": the prompt is processed in
+// parallel; Section 5.1.2 "Recomputation": a preempted request's prompt and generated tokens
+// are re-processed from scratch; Appendix B.1: prefill is scheduled in chunks).  Sequence b
+// contributes q_len_b = cu_q_lens[b+1] - cu_q_lens[b] query tokens, the last q_len_b of its
+// ctx_lens[b] cached tokens (their K/V are already in the cache).  Query i sits at position
+// pos = ctx_b - q_len_b + i and attends causally to cached tokens t <= pos:
+//     out[cu_q_lens[b] + i, h, :] = softmax_{t <= pos}(scale * <q, K_t>) . V_t
+// out: double [total_q, H, D].  Returns -1 on inconsistent lengths or a bad block id.
+int oracle_pa_prefill(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                      const int32_t* block_tables, int32_t max_blocks, const int32_t* ctx_lens,
+                      const int32_t* cu_q_lens, int32_t batch, int32_t H, int32_t Hkv, int32_t D,
+                      int32_t bs, int32_t num_blocks, int64_t stride_block, int64_t stride_head,
+                      int64_t stride_tok, double scale, double* out, int32_t num_threads) {
+    if (H % Hkv != 0) return -1;
+    const int G = H / Hkv;
+    if (batch > 0 && cu_q_lens[0] != 0) return -1;
+    for (int b = 0; b < batch; ++b) {
+        const int ql = cu_q_lens[b + 1] - cu_q_lens[b], L = ctx_lens[b];
+        if (ql < 0 || L < ql || L > static_cast<int64_t>(max_blocks) * bs) return -1;
+        for (int j = 0; j < (L + bs - 1) / bs; ++j) {
+            const int p = block_tables[static_cast<int64_t>(b) * max_blocks + j];
+            if (p < 0 || p >= num_blocks) return -1;
+        }
+    }
+    const int total_q = batch > 0 ? cu_q_lens[batch] : 0;
+    std::vector<int> seq_of(total_q);
+    for (int b = 0; b < batch; ++b)
+        for (int i = cu_q_lens[b]; i < cu_q_lens[b + 1]; ++i) seq_of[i] = b;
+    const int64_t rows = static_cast<int64_t>(total_q) * H;
+#ifdef _OPENMP
+    const int nt = oracle_threads(num_threads);
+#pragma omp parallel for schedule(dynamic, 1) num_threads(nt)
+#else
+    (void)num_threads;
+#endif
+    for (int64_t r = 0; r < rows; ++r) {
+        const int tok = static_cast<int>(r / H), h = static_cast<int>(r % H), kvh = h / G;
+        const int b = seq_of[tok];
+        const int ql = cu_q_lens[b + 1] - cu_q_lens[b];
+        const int pos = ctx_lens[b] - ql + (tok - cu_q_lens[b]);
+        const int n = pos + 1;  // visible cached tokens
+        double* o = out + r * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        const uint16_t* qrow = q + r * D;
+        const int32_t* table = block_tables + static_cast<int64_t>(b) * max_blocks;
+        std::vector<double> s(n);
+        for (int t = 0; t < n; ++t) {
+            const int64_t base = table[t / bs] * stride_block + kvh * stride_head +
+                                 (t % bs) * stride_tok;
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d)
+                acc += bf16_to_double(qrow[d]) * bf16_to_double(k_cache[base + d]);
+            s[t] = scale * acc;
+        }
+        double m = s[0];
+        for (int t = 1; t < n; ++t) m = s[t] > m ? s[t] : m;
+        double Z = 0.0;
+        for (int t = 0; t < n; ++t) {
+            s[t] = std::exp(s[t] - m);
+            Z += s[t];
+        }
+        for (int t = 0; t < n; ++t) {
+            const int64_t base = table[t / bs] * stride_block + kvh * stride_head +
+                                 (t % bs) * stride_tok;
+            const double w = s[t];
+            for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(v_cache[base + d]);
+        }
+        for (int d = 0; d < D; ++d) o[d] /= Z;
     }
     return 0;
 }
