@@ -183,6 +183,35 @@ int pa_decode_host(const pa_shape* shape, const void* q_host, const void* k_cach
                    size_t workspace_bytes, int32_t partition_tokens, int32_t* dev_status,
                    void* cuda_stream);
 
+/* Bytes of device workspace pa_prefill needs for at most `max_batch` sequences. */
+int pa_prefill_workspace_bytes(int32_t max_batch, size_t* bytes);
+
+/*
+ * Prefill / recomputation attention over the paged cache (Section 2.1 "Prefill"; Section
+ * 5.1.2 "Recomputation": a preempted request's prompt and generated tokens are re-processed;
+ * Appendix B.1: prefill runs in chunks under a token budget).  Sequence b contributes
+ * q_len_b = cu_q_lens[b+1] - cu_q_lens[b] query tokens: the last q_len_b of its ctx_lens[b]
+ * cached tokens, whose K/V must already be in the cache (kv_append).  Query i of sequence b
+ * sits at position pos = ctx_lens[b] - q_len_b + i and attends causally to tokens t <= pos:
+ *     out[cu_q_lens[b] + i, h, :] = softmax_{t <= pos}(scale * <q, K_t>) . V_t
+ *
+ *   q             dev bf16 [total_q, H, D] (tokens of all sequences packed), 16-byte aligned
+ *   k_cache, v_cache, block_tables, max_blocks_per_seq   as for pa_decode
+ *   ctx_lens      dev int32 [batch]: cached tokens visible to the last query of the chunk
+ *   cu_q_lens     dev int32 [batch + 1]: prefix sums of the query counts, cu_q_lens[0] = 0,
+ *                 cu_q_lens[batch] = total_q
+ *   out           dev bf16 [total_q, H, D]
+ *   workspace     dev, >= pa_prefill_workspace_bytes(batch), 256-byte aligned
+ *   dev_status    as for pa_decode: inconsistent lengths set PA_STATUS_BAD_SEQ_LEN (that
+ *                 sequence's rows are left unwritten), a bad used block id sets
+ *                 PA_STATUS_BAD_BLOCK_ID (affected rows are zero)
+ * Two kernels are enqueued (a one-CTA plan and the attention kernel).
+ */
+int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const void* v_cache,
+               const int32_t* block_tables, int32_t max_blocks_per_seq, const int32_t* ctx_lens,
+               const int32_t* cu_q_lens, int32_t batch, int32_t total_q, float scale, void* out,
+               void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
 /*
  * KV append (Section 2.2 "KV-Cache": with every decoding step the KV vectors of the newly
  * generated token are appended to the cache).  For every b < batch with slot_mapping[b] >= 0

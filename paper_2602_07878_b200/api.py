@@ -30,7 +30,8 @@ PA_STATIC_WORKSPACE_BYTES = 64 << 20
 EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
-           "pa_decode_static", "kv_append"]
+           "pa_decode_static", "kv_append",
+           "pa_prefill_workspace_bytes", "pa_prefill"]
 
 
 class PaShape(ctypes.Structure):
@@ -74,6 +75,11 @@ def lib() -> ctypes.CDLL:
         L.pa_decode_static.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, i64, ctypes.c_float,
                                        vp, i32, vp, vp]
         L.pa_decode_static.restype = ctypes.c_int
+        L.pa_prefill_workspace_bytes.argtypes = [i32, psz]
+        L.pa_prefill_workspace_bytes.restype = ctypes.c_int
+        L.pa_prefill.argtypes = [pshape, vp, vp, vp, vp, i32, vp, vp, i32, i32, ctypes.c_float, vp,
+                                 vp, sz, vp, vp]
+        L.pa_prefill.restype = ctypes.c_int
         L.kv_append.argtypes = [pshape, vp, vp, vp, vp, vp, i32, vp, vp]
         L.kv_append.restype = ctypes.c_int
         L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
@@ -265,3 +271,28 @@ def kv_append(k_cache, v_cache, k_new, v_new, slot_mapping, *, dev_status=None, 
                          _ptr(v_new), _ptr(slot_mapping), k_new.shape[0], _ptr(dev_status),
                          _stream(stream))
     _check(rc, "kv_append")
+
+
+def pa_prefill_workspace_bytes(max_batch: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().pa_prefill_workspace_bytes(max_batch, ctypes.byref(out)),
+           "pa_prefill_workspace_bytes")
+    return int(out.value)
+
+
+def pa_prefill(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, out, workspace, *,
+               dev_status=None, stream=None):
+    """Forward to pa_prefill.  q/out [total_q,H,D] bf16 (packed tokens); ctx_lens int32 [B];
+    cu_q_lens int32 [B+1]; caches and block_tables as for pa_decode."""
+    shape = shape_of(k_cache, q.shape[1])
+    assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
+    assert block_tables.dtype == torch.int32 and ctx_lens.dtype == torch.int32
+    assert cu_q_lens.dtype == torch.int32 and cu_q_lens.numel() == ctx_lens.numel() + 1
+    assert q.is_contiguous() and out.is_contiguous() and block_tables.is_contiguous()
+    rc = lib().pa_prefill(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                          _ptr(block_tables), block_tables.shape[1], _ptr(ctx_lens),
+                          _ptr(cu_q_lens), ctx_lens.numel(), q.shape[0], float(scale), _ptr(out),
+                          _ptr(workspace), workspace.numel() * workspace.element_size(),
+                          _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_prefill")
+    return out

@@ -1,5 +1,6 @@
 // Host/device declarations shared by the library's translation units (not installed).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -37,5 +38,11 @@ struct DeviceInfo {
 int get_device_info(DeviceInfo* info);
 
 int validate_shape(const pa_shape* s);
+
+// TMA tensor map over one layer's cache: dims (dim, slot, kv head, block), box 64 x 16 x 1 x 1,
+// 128-byte swizzle; block ids outside the pool are out of bounds and read as zeros.
+int make_cache_map(CUtensorMap* map, const void* base, const pa_shape* s);
+
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // bound of every in-kernel wait
 
 }  // namespace pk

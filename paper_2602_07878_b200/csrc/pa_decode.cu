@@ -21,6 +21,7 @@
 #include <utility>
 #include <vector>
 
+#include "attn_block.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -208,7 +209,6 @@ struct DecodeParams {
     float scale_log2;
 };
 
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
 template <int D, bool HI>
 struct UnitRegs {
@@ -320,19 +320,9 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         build(r1, k1, v1, U1);
     }
 
-    // ---- per-lane constants of the fragment addresses -------------------------------------
-    // K (B operand, not transposed): matrix i = lane>>3 -> tokens (i>>1)*8.., 16-byte chunk
-    // 2*ks + (i&1); V (B operand, transposed): tokens (i&1)*8.., chunk 2*jj + (i>>1).
-    const int mi = lane >> 3, mr = lane & 7;
-    const uint32_t k_row = ((mi >> 1) * 8 + mr) * 128;
-    const uint32_t k_cb = mi & 1;
-    const uint32_t v_row = ((mi & 1) * 8 + mr) * 128;
-    const uint32_t v_cb = mi >> 1;
-
-    float o[NT][4];
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+    AttnFrag<D, HI> A;
+    A.init_lane(lane);
+    A.reset();
 
     uint32_t n_issued = 0, n_done = 0;
     int iu = 0, ib = 0, cb = 0;  // issue cursor (unit 0/1, block), compute cursor
@@ -378,108 +368,16 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             const uint32_t kbase = slots + s * SLOT, vbase = kbase + TILE;
             const int nvalid = min(BS, U0.ntok - cb * BS);
 
-            if (nvalid < BS) {
-                // unused slots of a sequence's last block may hold anything: zero their V rows
-                // (0 * NaN would poison the accumulators); their scores are masked below
-                const int nchunk = (BS - nvalid) * 8;
-                for (int hf = 0; hf < HALVES; ++hf)
-                    for (int c = lane; c < nchunk; c += 32)
-                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(
-                                         vbase + hf * HALF_BYTES + nvalid * 128 + c * 16),
-                                     "r"(0u)
-                                     : "memory");
-                fence_proxy_async_smem();
-                __syncwarp();
-            }
-
-            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens
-            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                uint32_t b00, b01, b10, b11;
-                const uint32_t chunk = ((ks & 3) * 2 + k_cb) ^ mr;
-                ldmatrix_x4(kbase + (ks >> 2) * HALF_BYTES + k_row + (chunk << 4), b00, b01, b10,
-                            b11);
-                const uint32_t a0 = U0.qa[ks][0], a2 = U0.qa[ks][QW == 4 ? 2 : 1];
-                const uint32_t a1 = HI ? U0.qa[ks][1] : 0u, a3 = HI ? U0.qa[ks][QW - 1] : 0u;
-                mma_bf16_16816(s0, a0, a1, a2, a3, b00, b01);
-                mma_bf16_16816(s1, a0, a1, a2, a3, b10, b11);
-            }
-
-            // scale to log2 units, mask tokens past the sequence end
-            const int c0 = 2 * t;
-            const bool v00 = c0 < nvalid, v01 = c0 + 1 < nvalid, v10 = c0 + 8 < nvalid,
-                       v11 = c0 + 9 < nvalid;
-            s0[0] = v00 ? s0[0] * sl2 : -INFINITY;
-            s0[1] = v01 ? s0[1] * sl2 : -INFINITY;
-            s1[0] = v10 ? s1[0] * sl2 : -INFINITY;
-            s1[1] = v11 ? s1[1] * sl2 : -INFINITY;
-            float mx0 = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-            const float mn0 = fmaxf(m0, mx0);
-            const float mu0 = mn0 == -INFINITY ? 0.f : mn0;
-            const float corr0 = ex2(m0 - mu0);
-            m0 = mn0;
-            const uint32_t pa0 = pack_bf16x2(ex2(s0[0] - mu0), ex2(s0[1] - mu0));
-            const uint32_t pa2 = pack_bf16x2(ex2(s1[0] - mu0), ex2(s1[1] - mu0));
-            // the row sum uses the rounded weights, the same ones the MMA multiplies by
-            l0 = l0 * corr0 + ((bf16lo_to_f32(pa0) + bf16hi_to_f32(pa0)) +
-                               (bf16lo_to_f32(pa2) + bf16hi_to_f32(pa2)));
-            uint32_t pa1 = 0u, pa3 = 0u;
-            float corr1 = 1.f;
-            if (HI) {
-                s0[2] = v00 ? s0[2] * sl2 : -INFINITY;
-                s0[3] = v01 ? s0[3] * sl2 : -INFINITY;
-                s1[2] = v10 ? s1[2] * sl2 : -INFINITY;
-                s1[3] = v11 ? s1[3] * sl2 : -INFINITY;
-                float mx1 = fmaxf(fmaxf(s0[2], s0[3]), fmaxf(s1[2], s1[3]));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                const float mn1 = fmaxf(m1, mx1);
-                const float mu1 = mn1 == -INFINITY ? 0.f : mn1;
-                corr1 = ex2(m1 - mu1);
-                m1 = mn1;
-                pa1 = pack_bf16x2(ex2(s0[2] - mu1), ex2(s0[3] - mu1));
-                pa3 = pack_bf16x2(ex2(s1[2] - mu1), ex2(s1[3] - mu1));
-                l1 = l1 * corr1 + ((bf16lo_to_f32(pa1) + bf16hi_to_f32(pa1)) +
-                                   (bf16lo_to_f32(pa3) + bf16hi_to_f32(pa3)));
-            }
-            // rescale only when some row's maximum moved (warp-uniform branch)
-            if (__any_sync(0xffffffffu, corr0 != 1.f || corr1 != 1.f)) {
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    o[nt][0] *= corr0;
-                    o[nt][1] *= corr0;
-                    if (HI) {
-                        o[nt][2] *= corr1;
-                        o[nt][3] *= corr1;
-                    }
-                }
-            }
-
-            // O += P V: V^T fragments straight from the [token][dim] tile
-#pragma unroll
-            for (int jj = 0; jj < D / 16; ++jj) {
-                uint32_t v0, v1, v2, v3;
-                const uint32_t chunk = ((jj & 3) * 2 + v_cb) ^ mr;
-                ldmatrix_x4_trans(vbase + (jj >> 2) * HALF_BYTES + v_row + (chunk << 4), v0, v1,
-                                  v2, v3);
-                mma_bf16_16816(o[2 * jj], pa0, pa1, pa2, pa3, v0, v1);
-                mma_bf16_16816(o[2 * jj + 1], pa0, pa1, pa2, pa3, v2, v3);
-            }
+            A.attend(kbase, vbase, U0.qa, nvalid, nvalid, nvalid, sl2, lane);
             ++n_done;
             ++cb;
         }
 
         // ---- unit finished: write its result, move to the next unit -----------------------------
         if (cb == U0.nblk) {
-            l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-            l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-            if (HI) {
-                l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-                l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-            }
+            A.reduce_row_sums();
+            const float l0 = A.l0, l1 = A.l1, m0 = A.m0, m1 = A.m1;
+            auto& o = A.o;
             const int h0 = U0.kvh * G + g;
             if (U0.direct) {
                 const float i0 = U0.bad ? 0.f : 1.f / l0, i1 = U0.bad ? 0.f : 1.f / l1;
@@ -521,10 +419,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
             if (iu == 1) iu = 0; else ib = 0;  // the issue cursor stays where it was
             cb = 0;
-            m0 = m1 = -INFINITY;
-            l0 = l1 = 0.f;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+            A.reset();
         }
     }
 }
@@ -652,7 +547,7 @@ static EncodeTiledFn get_encode_fn() {
 }
 
 // tensor map over one layer's cache: dims (dim, slot, kv head, block), box 64 x 16 x 1 x 1
-static int make_cache_map(CUtensorMap* map, const void* base, const pa_shape* s) {
+int make_cache_map(CUtensorMap* map, const void* base, const pa_shape* s) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) {
         set_cuda_error((int)cudaErrorSymbolNotFound);

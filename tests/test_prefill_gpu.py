@@ -1,0 +1,95 @@
+"""GPU parity of pa_prefill (through the C-ABI) against the fp64 prefill oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_07878_b200 import api
+from paper_2602_07878_b200 import workloads as wl
+from helpers import assert_parity, bits_to_torch, torch_to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+class GpuPrefill:
+    def __init__(self, spec, q_bits, k_bits, v_bits):
+        self.spec = spec
+        self.q = bits_to_torch(q_bits)
+        self.k, self.v = bits_to_torch(k_bits), bits_to_torch(v_bits)
+        self.tables = torch.from_numpy(spec.block_tables).cuda()
+        self.ws = torch.empty(api.pa_prefill_workspace_bytes(spec.batch), dtype=torch.uint8,
+                              device="cuda")
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def run(self, ctx, cu, q=None, tables=None):
+        q = self.q if q is None else q
+        out = torch.full_like(q, float("nan"))
+        api.pa_prefill(q, self.k, self.v, self.tables if tables is None else tables,
+                       torch.from_numpy(np.asarray(ctx, np.int32)).cuda(),
+                       torch.from_numpy(np.asarray(cu, np.int32)).cuda(), self.spec.scale, out,
+                       self.ws, dev_status=self.status)
+        torch.cuda.synchronize()
+        return out
+
+
+def make_case(ctx, qlens, H, Hkv, D, seed):
+    spec = wl.make_spec("t", seq_lens=ctx, num_q_heads=H, num_kv_heads=Hkv, head_dim=D,
+                        occupancy=0.85, seed=seed)
+    k, v = wl.pools_np(spec)
+    cu = np.concatenate([[0], np.cumsum(qlens)]).astype(np.int32)
+    q = wl.normal_bf16_np(0, int(cu[-1]) * H * D, 700 + seed).reshape(int(cu[-1]), H, D)
+    return spec, q, k, v, cu
+
+
+@pytest.mark.parametrize("H,Hkv,D", [(8, 8, 64), (8, 2, 128), (32, 8, 128), (16, 1, 128),
+                                     (6, 2, 64), (10, 2, 128), (8, 1, 64)])
+def test_mixed_chunks_match_oracle(H, Hkv, D):
+    ctx = [37, 64, 5, 130, 1, 700, 16, 333]
+    qlens = [37, 10, 0, 33, 1, 512, 16, 1]
+    spec, q, k, v, cu = make_case(ctx, qlens, H, Hkv, D, seed=H + Hkv + D)
+    g = GpuPrefill(spec, q, k, v)
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, f"H{H}/{Hkv} D{D}")
+
+
+def test_single_query_token_equals_decode_bits():
+    # a chunk of one query token per sequence is a decode step
+    spec, q, k, v, cu = make_case([90, 17, 256], [1, 1, 1], 8, 2, 128, seed=9)
+    g = GpuPrefill(spec, q, k, v)
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    ref = oracle.pa_decode(q, k, v, spec.block_tables, spec.seq_lens, spec.scale)
+    assert_parity(out, ref)
+
+
+def test_chunked_recompute_of_a_long_sequence():
+    """Recompute a 3000-token victim in 512-token chunks; every chunk sees the cache up to its
+    own end.  The concatenation equals the one-shot oracle."""
+    spec, q, k, v, cu = make_case([3000], [3000], 32, 8, 128, seed=10)
+    g = GpuPrefill(spec, q, k, v)
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    outs = []
+    for start in range(0, 3000, 512):
+        end = min(3000, start + 512)
+        outs.append(g.run([end], [0, end - start], q=g.q[start:end].contiguous()))
+    assert int(g.status.item()) == 0
+    assert_parity(torch_to_f64(torch.cat(outs)), ref, "chunked recompute")
+
+
+def test_bad_lengths_and_ids_are_reported():
+    spec, q, k, v, cu = make_case([40, 64], [8, 16], 8, 2, 128, seed=11)
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    g = GpuPrefill(spec, q, k, v)
+    out = torch_to_f64(g.run([4, 64], cu))           # ctx < q_len for sequence 0
+    assert int(g.status.item()) == api.PA_STATUS_BAD_SEQ_LEN
+    assert np.isnan(out[:8]).all()                   # rows of the refused sequence untouched
+    assert_parity(out[8:], ref[8:])
+    g.status.zero_()
+    t = spec.block_tables.copy()
+    t[1, 2] = spec.num_blocks + 5
+    out = torch_to_f64(g.run(spec.seq_lens, cu, tables=torch.from_numpy(t).cuda()))
+    assert int(g.status.item()) == api.PA_STATUS_BAD_BLOCK_ID
+    assert_parity(out[:8], ref[:8])
+    # queries at positions 48..63 need block 2 (tokens 32..47): all of sequence 1's rows are zero
+    assert (out[8:] == 0).all()
