@@ -397,6 +397,8 @@ def run_ours(args):
 
     if rank == 0 and world == 1:
         line["kv_append"] = bench_append(torch, api, spec, k, v)
+        if not args.no_recompute:
+            line["recompute"] = bench_recompute(torch, api, spec, k, v, tables)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -434,6 +436,52 @@ def bench_append(torch, api, spec, k, v, calls=200):
     us = e0.elapsed_time(e1) * 1e3 / calls
     return {"us_per_call": us, "tokens": int(len(rows)), "bytes": nbytes,
             "gbps": nbytes / us / 1e3, "bound": "launch latency / host issue rate (2 MB moved per call)"}
+
+
+def bench_recompute(torch, api, spec, k, v, tables, chunk=512):
+    """Recomputation recovery of the longest sequence of the batch: causal prefill attention
+    over its cached tokens in chunks of `chunk` query tokens (one pa_prefill call per chunk,
+    context growing).  A dense contraction: reported in TFLOP/s against the bf16 tensor peak."""
+    b = int(np.argmax(spec.seq_lens))
+    L = int(spec.seq_lens[b])
+    H, D = spec.num_q_heads, spec.head_dim
+    q = torch.empty(L, H, D, dtype=torch.bfloat16, device="cuda").normal_()
+    out = torch.empty_like(q)
+    tab = tables[b:b + 1].contiguous()
+    ws = torch.empty(api.pa_prefill_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    calls = []
+    for start in range(0, L, chunk):
+        end = min(L, start + chunk)
+        calls.append((start, end, torch.tensor([end], dtype=torch.int32, device="cuda"),
+                      torch.tensor([0, end - start], dtype=torch.int32, device="cuda")))
+
+    def run():
+        for start, end, ctx, cu in calls:
+            api.pa_prefill(q[start:end], k, v, tab, ctx, cu, spec.scale, out[start:end], ws,
+                           dev_status=status)
+
+    run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    run()
+    e1.record()
+    e1.synchronize()
+    ms = e0.elapsed_time(e1)
+    # 4 * D flops per (query, visible key, head): QK^T and PV, 2 flops per multiply-add
+    pairs = sum((end - start) * (start + end + 1) // 2 for start, end, _, _ in calls)
+    flops = 4.0 * D * H * pairs
+    peak = None
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            peak = float(json.load(f)["bf16_tflops"])
+    assert int(status.item()) == 0
+    return {"tokens": L, "chunk": chunk, "calls": len(calls), "ms": ms, "tflops": flops / ms / 1e9,
+            "bound": "tensor", "peak_tflops": peak,
+            "frac": (flops / ms / 1e9 / peak) if peak else None,
+            "tokens_per_s": L / (ms / 1e3)}
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pa_decode_kernel launch, from the ncu
@@ -672,6 +720,7 @@ def main():
     ap.add_argument("--churn-steps", type=int, default=3)
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-recompute", action="store_true")
     ap.add_argument("--cpu-fraction", type=float, default=1.0,
                     help="fraction of the batch's tokens the CPU baseline pass covers")
     ap.add_argument("--swap-pool-blocks", type=int, default=6144)
