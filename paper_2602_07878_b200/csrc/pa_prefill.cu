@@ -7,7 +7,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
 #include <mutex>
+#include <string>
 
 #include "attn_block.cuh"
 #include "internal.h"
@@ -256,6 +258,382 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
     return check_cuda(cudaLaunchKernelEx(&cfg, kern, km, vm, pp));
 }
 
+
+// ======================================================================================
+// tcgen05 version: one CTA = 128 query rows ((token, head) pairs of one KV-head group)
+// ======================================================================================
+// Warps 0-3: softmax and epilogue (thread i owns row i = TMEM lane i); warp 4: TMA producer;
+// warp 5: MMA issuer.  Per 64-token KV step:  S = Q K^T (M 128, N 64, K 128) into one of two
+// TMEM score buffers, the softmax warps turn S into bf16 weights P in shared memory (and
+// rescale the TMEM accumulator O when a row maximum has grown by more than 2^8), then
+// O += P V (M 128, N 128, K 64).  Score buffers, P buffers and four KV stages are
+// double/quad buffered so that Q K^T of step j+1 overlaps the softmax of step j.
+namespace tc {
+constexpr int ROWS = 128, STEP = 64, ST = 4, D = 128;
+constexpr int Q_BYTES = ROWS * D * 2;                 // two 64-dim halves of 128 rows x 128 B
+constexpr int KV_HALF = STEP * 128;                   // 64 tokens x 128 B
+constexpr int STAGE_BYTES = 4 * KV_HALF;              // K half 0, K half 1, V half 0, V half 1
+constexpr int P_BYTES = ROWS * STEP * 2;              // 128 rows x 64 tokens bf16
+constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + ST * STAGE_BYTES;
+constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
+// barriers (8 bytes each)
+enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + ST, B_SFULL = B_KVEMPTY + ST,
+       B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2, B_COUNT = B_PVDONE + 2 };
+constexpr int OFF_MISC = OFF_BAR + B_COUNT * 8;       // tmem base, abort flag, bad flag
+constexpr int SMEM_BYTES = OFF_MISC + 64 + 1024;      // + slack for 1024-byte alignment
+constexpr int TMEM_COLS = 256;                        // S0 [0,64) S1 [64,128) O [128,256)
+}  // namespace tc
+
+struct PrefillTcParams {
+    PrefillParams base;
+    int tokens_per_tile;  // 128 / G
+};
+
+__global__ void __launch_bounds__(192, 1)
+pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
+                     const __grid_constant__ CUtensorMap kmap,
+                     const __grid_constant__ CUtensorMap vmap, const PrefillTcParams tp) {
+    using namespace tc;
+    const PrefillParams& p = tp.base;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gbase = smem_raw + (sbase - smem_u32(smem_raw));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    auto bar = [&](int i) { return sbase + OFF_BAR + 8 * i; };
+    volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + OFF_MISC);
+    // misc[0] = TMEM base address, misc[1] = abort flag, misc[2] = bad block id seen
+
+    pdl_launch_dependents();
+    pdl_wait();
+
+    // ---- which tile -------------------------------------------------------------------------
+    const int G = p.G, H = p.H, Hkv = p.Hkv, tpt = tp.tokens_per_tile;
+    const int n_units = p.hdr[PF_N_GROUPS] * Hkv;
+    if ((int)blockIdx.x >= n_units) return;
+    const int u = n_units - 1 - blockIdx.x;  // later tiles see more tokens: start them first
+    const int gi = u / Hkv, kvh = u - gi * Hkv;
+    int lo = 0, hi = p.batch;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (p.gstart[mid] <= gi) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int q0 = p.cu_q_lens[b], ql = p.cu_q_lens[b + 1] - q0, L = p.ctx_lens[b];
+    const int tok0 = (gi - p.gstart[b]) * tpt;
+    const int ntok = min(tpt, ql - tok0);
+    const int pos_max = L - ql + tok0 + ntok - 1;
+    const int n_steps = pos_max / STEP + 1;
+    const int nblk_seq = (L + BS - 1) / BS;
+
+    if (tid == 0) {
+        mbar_init(bar(B_QFULL), 1);
+        for (int i = 0; i < ST; ++i) mbar_init(bar(B_KVFULL + i), 1), mbar_init(bar(B_KVEMPTY + i), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(B_SFULL + i), 1);
+            mbar_init(bar(B_SFREE + i), 4);
+            mbar_init(bar(B_PFULL + i), 4);
+            mbar_init(bar(B_PVDONE + i), 1);
+        }
+        mbar_init_fence();
+        misc[1] = 0;
+        misc[2] = 0;
+    }
+    if (warp == 5) tmem_alloc(sbase + OFF_MISC, TMEM_COLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = misc[0];
+
+    // every wait is bounded; a wait that gives up raises the abort flag and everyone leaves
+    auto wait = [&](int b_idx, uint32_t parity) -> bool {
+        if (misc[1]) return false;
+        if (mbar_wait_bounded(bar(b_idx), parity, WAIT_LIMIT_NS)) return true;
+        misc[1] = 1;
+        atomicOr(p.status, PA_STATUS_TIMEOUT);
+        return false;
+    };
+
+    if (warp == 4) {
+        // ===================== TMA producer =====================
+        if (lane == 0) {
+            tma_prefetch_desc(&qmap);
+            tma_prefetch_desc(&kmap);
+            tma_prefetch_desc(&vmap);
+            mbar_arrive_expect_tx(bar(B_QFULL), Q_BYTES);
+            tma_load_4d(sbase + OFF_Q, &qmap, bar(B_QFULL), 0, 0, kvh, q0 + tok0);
+            tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &qmap, bar(B_QFULL), 64, 0, kvh, q0 + tok0);
+        }
+        const int32_t* table = p.block_tables + (size_t)b * p.max_blocks;
+        int ids = lane < nblk_seq ? __ldg(&table[lane]) : p.NB;
+        int ids_next = 32 + lane < nblk_seq ? __ldg(&table[32 + lane]) : p.NB;
+        for (int j = 0; j < n_steps; ++j) {
+            const int stage = j % ST;
+            if (j >= ST && !wait(B_KVEMPTY + stage, ((j / ST) - 1) & 1)) break;
+            const int blk0 = j * 4;
+            if (blk0 > 0 && (blk0 & 31) == 0) {
+                ids = ids_next;
+                ids_next = blk0 + 32 + lane < nblk_seq ? __ldg(&table[blk0 + 32 + lane]) : p.NB;
+            }
+            // lane l < 16: block l>>2 of the step, tile l&3 (K half 0/1, V half 0/1)
+            const int id = __shfl_sync(0xffffffffu, ids, (blk0 + (lane >> 2)) & 31);
+            const bool used = blk0 + (lane >> 2) < nblk_seq;
+            if (used && (unsigned)id >= (unsigned)p.NB && (lane & 3) == 0) {
+                misc[2] = 1;
+                atomicOr(p.status, PA_STATUS_BAD_BLOCK_ID);
+            }
+            if (lane == 0) mbar_arrive_expect_tx(bar(B_KVFULL + stage), STAGE_BYTES);
+            __syncwarp();
+            if (lane < 16) {
+                const int which = lane & 3;
+                const uint32_t dst = sbase + OFF_KV + stage * STAGE_BYTES + which * KV_HALF +
+                                     (lane >> 2) * (BS * 128);
+                // an id outside the pool is out of the tensor's bounds and reads as zeros
+                tma_load_4d(dst, which < 2 ? &kmap : &vmap, bar(B_KVFULL + stage), (which & 1) * 64,
+                            0, kvh, used ? id : p.NB);
+            }
+        }
+    } else if (warp == 5) {
+        // ===================== MMA issuer (one thread) =====================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = tc_idesc_bf16(ROWS, STEP, false);
+            constexpr uint32_t idesc_pv = tc_idesc_bf16(ROWS, D, true);
+            bool ok = wait(B_QFULL, 0);
+            for (int j = 0; ok && j <= n_steps; ++j) {
+                if (j < n_steps) {  // S[j % 2] = Q K_j^T
+                    const int stage = j % ST;
+                    ok = wait(B_KVFULL + stage, (j / ST) & 1);
+                    if (ok && j >= 2) ok = wait(B_SFREE + (j & 1), ((j >> 1) - 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t kb = sbase + OFF_KV + stage * STAGE_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint64_t a = tc_smem_desc(
+                            sbase + OFF_Q + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32, 16, 1024);
+                        const uint64_t bd =
+                            tc_smem_desc(kb + (ks >> 2) * KV_HALF + (ks & 3) * 32, 16, 1024);
+                        tc_mma_bf16(tmem + (j & 1) * STEP, a, bd, idesc_qk, ks > 0);
+                    }
+                    tc_commit(bar(B_SFULL + (j & 1)));
+                }
+                if (j >= 1) {  // O += P_{j-1} V_{j-1}
+                    const int i = j - 1, stage = i % ST;
+                    ok = wait(B_PFULL + (i & 1), (i >> 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t vb = sbase + OFF_KV + stage * STAGE_BYTES + 2 * KV_HALF;
+                    const uint32_t pb = sbase + OFF_P + (i & 1) * P_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < STEP / 16; ++kk) {
+                        const uint64_t a = tc_smem_desc(pb + kk * 32, 16, 1024);
+                        // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
+                        const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
+                        tc_mma_bf16(tmem + 2 * STEP, a, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar(B_KVEMPTY + stage));
+                    tc_commit(bar(B_PVDONE + (i & 1)));
+                }
+            }
+        }
+    } else {
+        // ===================== softmax + epilogue: thread = row =====================
+        const int row = tid;
+        const int tk = row / G, hd = row - tk * G;
+        const bool row_ok = tk < ntok;
+        const int pos = row_ok ? L - ql + tok0 + tk : 0x7fffffff;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const float sl2 = p.scale_log2;
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_steps; ++j) {
+            ok = wait(B_SFULL + (j & 1), (j >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            uint32_t sr[2][32];
+            tmem_ld32(tmem + lane_base + (j & 1) * STEP, sr[0]);
+            tmem_ld32(tmem + lane_base + (j & 1) * STEP + 32, sr[1]);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_SFREE + (j & 1)));
+
+            const int t0 = j * STEP;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < STEP; ++c) {
+                float v = __uint_as_float(sr[c >> 5][c & 31]) * sl2;
+                v = (t0 + c <= pos) ? v : -INFINITY;
+                sr[c >> 5][c & 31] = __float_as_uint(v);
+                mx = fmaxf(mx, v);
+            }
+            // keep the reference maximum unless it would let a weight exceed 2^8
+            float corr = 1.f;
+            if (mx > m_ref + 8.f) {
+                corr = ex2(m_ref - mx);  // 0 on the first step
+                m_ref = mx;
+            }
+            const float mu = m_ref == -INFINITY ? 0.f : m_ref;
+            uint32_t pk[STEP / 2];
+            float lsum = 0.f;
+#pragma unroll
+            for (int c = 0; c < STEP; c += 2) {
+                const uint32_t w = pack_bf16x2(ex2(__uint_as_float(sr[c >> 5][c & 31]) - mu),
+                                               ex2(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]) - mu));
+                pk[c >> 1] = w;
+                lsum += bf16lo_to_f32(w) + bf16hi_to_f32(w);
+            }
+            l = l * corr + lsum;
+
+            // the P buffer of step j-2 must have been consumed
+            if (j >= 2) {
+                ok = wait(B_PVDONE + (j & 1), ((j >> 1) - 1) & 1);
+                if (!ok) break;
+            }
+            // rescale O (only after the first step, and only once P V of step j-1 is complete)
+            if (j >= 1 && __any_sync(0xffffffffu, corr != 1.f)) {
+                ok = wait(B_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+#pragma unroll 1
+                for (int c = 0; c < D; c += 32) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem + lane_base + 2 * STEP + c, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+                    tmem_st32(tmem + lane_base + 2 * STEP + c, o);
+                }
+                tmem_wait_st();
+            }
+            // P row -> shared memory, 128-byte swizzle (16-byte chunk c of row r at c ^ (r & 7))
+            {
+                const uint32_t prow = sbase + OFF_P + (j & 1) * P_BYTES + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(
+                                     prow + ((c ^ (row & 7)) << 4)),
+                                 "r"(pk[4 * c]), "r"(pk[4 * c + 1]), "r"(pk[4 * c + 2]),
+                                 "r"(pk[4 * c + 3])
+                                 : "memory");
+            }
+            // slots past the end of the sequence may hold anything: zero their V rows
+            if (t0 + STEP > L) {
+                ok = wait(B_KVFULL + (j % ST), (j / ST) & 1);
+                if (!ok) break;
+                const int r0 = max(0, L - t0);                      // first unused row of the step
+                const int r1 = min(STEP, ((L + BS - 1) / BS) * BS - t0);  // end of the partial block
+                const uint32_t vb = sbase + OFF_KV + (j % ST) * STAGE_BYTES + 2 * KV_HALF;
+                for (int e = tid; e < (r1 - r0) * 16; e += 128) {
+                    const int r = r0 + (e >> 4), c = e & 15;  // 16 chunks: 8 per half
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(
+                                     vb + (c >> 3) * KV_HALF + r * 128 + (c & 7) * 16),
+                                 "r"(0u)
+                                 : "memory");
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_PFULL + (j & 1)));
+        }
+        // ---- epilogue: O / l -> bf16 rows ----
+        if (ok) ok = wait(B_PVDONE + ((n_steps - 1) & 1), ((n_steps - 1) >> 1) & 1);
+        if (ok) {
+            tc_fence_after_sync();
+            const bool bad = misc[2] != 0;
+            const float inv = bad ? 0.f : 1.f / l;
+            __nv_bfloat16* dst =
+                p.out + ((size_t)(q0 + tok0 + tk) * H + (size_t)kvh * G + hd) * D;
+#pragma unroll 1
+            for (int c = 0; c < D; c += 32) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_base + 2 * STEP + c, o);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 w;
+                        w.x = bad ? 0u : pack_bf16x2(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+                        w.y = bad ? 0u : pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                        w.z = bad ? 0u : pack_bf16x2(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                        w.w = bad ? 0u : pack_bf16x2(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                        *reinterpret_cast<uint4*>(dst + c + i) = w;
+                    }
+                }
+            }
+        }
+    }
+    // ---- teardown: everyone meets, then the allocating warp returns the tensor memory ----
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+}
+
+// tensor map over the packed queries viewed as [total_q][Hkv][G][D]: box 64 x G x 1 x (128/G)
+static int make_q_map(CUtensorMap* map, const void* q, int total_q, int Hkv, int G, int D) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                 const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                 const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn enc = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
+                cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            enc = reinterpret_cast<EncodeFn>(ptr);
+    });
+    if (!enc) {
+        set_cuda_error((int)cudaErrorSymbolNotFound);
+        return PA_ERR_CUDA;
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)G, (cuuint64_t)Hkv, (cuuint64_t)total_q};
+    cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)G * D * 2, (cuuint64_t)Hkv * G * D * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)G, 1, (cuuint32_t)(128 / G)};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error((int)r);
+        return PA_ERR_CUDA;
+    }
+    return PA_OK;
+}
+
+static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
+                             const PrefillTcParams& tp, int max_tiles, const DeviceInfo& dev,
+                             cudaStream_t st) {
+    static int configured_dev = -1;
+    static std::mutex mu;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (configured_dev != dev.device) {
+            int rc = check_cuda(cudaFuncSetAttribute(pa_prefill_tc_kernel,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     tc::SMEM_BYTES));
+            if (rc) return rc;
+            configured_dev = dev.device;
+        }
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(max_tiles);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = tc::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    count_launch();
+    return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_tc_kernel, qm, km, vm, tp));
+}
+
 }  // namespace pk
 
 using namespace pk;
@@ -306,7 +684,13 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
     plan.batch = batch;
     plan.max_blocks = max_blocks_per_seq;
     plan.total_q = total_q;
-    plan.tpg = 16 / G;
+    // tensor-core path: 128-row tiles; needs head_dim 128 and a group size that divides 128
+    static const bool force_mma = [] {
+        const char* e = std::getenv("PAGEDKV_PREFILL");
+        return e && std::string(e) == "mma";
+    }();
+    const bool use_tc = !force_mma && shape->head_dim == 128 && (128 % G) == 0;
+    plan.tpg = use_tc ? 128 / G : 16 / G;
     plan.hdr = hdr;
     plan.gstart = hdr + PF_WORDS;
     plan.status = dev_status ? dev_status : hdr + PF_STATUS;
@@ -332,6 +716,16 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
     pp.NB = shape->num_blocks;
     pp.tpg = plan.tpg;
     pp.scale_log2 = scale * 1.4426950408889634f;
+    if (use_tc) {
+        CUtensorMap qm;
+        rc = make_q_map(&qm, q, total_q, pp.Hkv, G, shape->head_dim);
+        if (rc) return rc;
+        PrefillTcParams tp;
+        tp.base = pp;
+        tp.tokens_per_tile = plan.tpg;
+        const int max_tiles = (total_q / plan.tpg + batch) * pp.Hkv;
+        return launch_prefill_tc(qm, km, vm, tp, max_tiles, dev, st);
+    }
     return shape->head_dim == 128 ? launch_prefill<128>(km, vm, pp, dev, st)
                                   : launch_prefill<64>(km, vm, pp, dev, st);
 }
