@@ -13,12 +13,12 @@ ABS_TOL = 1e-2
 REL_TOL = 2e-2
 
 
-def assert_parity(gpu: np.ndarray, ref: np.ndarray, what: str = ""):
+def assert_parity(gpu: np.ndarray, ref: np.ndarray, what: str = "", abs_tol: float = ABS_TOL):
     gpu = np.asarray(gpu, dtype=np.float64)
     assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
     assert np.isfinite(gpu).all(), f"{what}: non-finite output"
     err = np.abs(gpu - ref)
-    assert err.max(initial=0.0) <= ABS_TOL, f"{what}: abs err {err.max():.3e}"
+    assert err.max(initial=0.0) <= abs_tol, f"{what}: abs err {err.max():.3e}"
     row_err = err.reshape(-1, err.shape[-1]).max(axis=1)
     row_ref = np.abs(ref).reshape(-1, ref.shape[-1]).max(axis=1)
     rel = row_err / np.maximum(row_ref, 1e-30)

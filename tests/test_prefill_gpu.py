@@ -42,7 +42,8 @@ def make_case(ctx, qlens, H, Hkv, D, seed):
 
 
 @pytest.mark.parametrize("H,Hkv,D", [(8, 8, 64), (8, 2, 128), (32, 8, 128), (16, 1, 128),
-                                     (6, 2, 64), (10, 2, 128), (8, 1, 64)])
+                                     (6, 2, 64), (10, 2, 128), (8, 1, 64), (4, 4, 128),
+                                     (8, 4, 128), (8, 1, 128), (64, 8, 128)])
 def test_mixed_chunks_match_oracle(H, Hkv, D):
     ctx = [37, 64, 5, 130, 1, 700, 16, 333]
     qlens = [37, 10, 0, 33, 1, 512, 16, 1]
@@ -93,3 +94,29 @@ def test_bad_lengths_and_ids_are_reported():
     assert_parity(out[:8], ref[:8])
     # queries at positions 48..63 need block 2 (tokens 32..47): all of sequence 1's rows are zero
     assert (out[8:] == 0).all()
+
+
+@pytest.mark.parametrize("H,Hkv", [(4, 4), (32, 8)])
+def test_long_context_chunks_with_ragged_ends(H, Hkv):
+    # chunks whose ends are not multiples of the kernels' 16/64/128-token tiles, contexts
+    # that end inside a block, several sequences of very different length in one call
+    ctx = [4999, 130, 1031, 64]
+    qlens = [517, 130, 7, 1]
+    spec, q, k, v, cu = make_case(ctx, qlens, H, Hkv, 128, seed=40 + H)
+    g = GpuPrefill(spec, q, k, v)
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, f"H{H}/{Hkv}")
+
+
+def test_large_scores_and_growing_maxima():
+    # scale 8 makes the running row maximum jump by far more than 2^8 between steps
+    spec, q, k, v, cu = make_case([700], [300], 8, 2, 128, seed=50)
+    g = GpuPrefill(spec, q, k, v)
+    spec.scale = np.float32(8.0)
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, 8.0)
+    # the softmax is nearly one-hot here, so outputs are single V rows of magnitude 2-4 where
+    # one bf16 step is 2^-6 = 0.0156: the absolute bound is widened to 2e-2 for this case only
+    assert_parity(out, ref, "scale 8", abs_tol=2e-2)
