@@ -48,14 +48,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Wait for a phase with a wall-clock bound.  Returns false if `limit_ns` passed first.
+// Wait for a phase with a wall-clock bound.  Returns false if `limit_ns` passed first.  The
+// clock is only looked at every 256 polls: reading it is slow, and a wait that is about to
+// succeed should not pay for it.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
                                                   unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    while (true) {
+    unsigned long long t0 = 0;
+    for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > limit_ns) return false;
+        if ((it & 255u) == 0u) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0)
+                t0 = now;
+            else if (now - t0 > limit_ns)
+                return false;
+        }
     }
 }
 
