@@ -458,29 +458,60 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             if (lane == 0) mbar_arrive(bar(B_SFREE + (j & 1)));
 
             const int t0 = j * STEP;
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < STEP; ++c) {
-                float v = __uint_as_float(sr[c >> 5][c & 31]) * sl2;
-                v = (t0 + c <= pos) ? v : -INFINITY;
-                sr[c >> 5][c & 31] = __float_as_uint(v);
-                mx = fmaxf(mx, v);
-            }
-            // keep the reference maximum unless it would let a weight exceed 2^8
-            float corr = 1.f;
-            if (mx > m_ref + 8.f) {
-                corr = ex2(m_ref - mx);  // 0 on the first step
-                m_ref = mx;
-            }
-            const float mu = m_ref == -INFINITY ? 0.f : m_ref;
             uint32_t pk[STEP / 2];
-            float lsum = 0.f;
+            float corr = 1.f, lsum = 0.f;
+            if (sl2 > 0.f) {
+                // fast path: maximum on the raw scores, one FMA + one EX2 per element
+                float mxr = -INFINITY;
+                if (__any_sync(0xffffffffu, t0 + STEP - 1 > pos)) {  // diagonal step: mask
 #pragma unroll
-            for (int c = 0; c < STEP; c += 2) {
-                const uint32_t w = pack_bf16x2(ex2(__uint_as_float(sr[c >> 5][c & 31]) - mu),
-                                               ex2(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]) - mu));
-                pk[c >> 1] = w;
-                lsum += bf16lo_to_f32(w) + bf16hi_to_f32(w);
+                    for (int c = 0; c < STEP; ++c) {
+                        float v = __uint_as_float(sr[c >> 5][c & 31]);
+                        v = (t0 + c <= pos) ? v : -INFINITY;
+                        sr[c >> 5][c & 31] = __float_as_uint(v);
+                        mxr = fmaxf(mxr, v);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < STEP; ++c)
+                        mxr = fmaxf(mxr, __uint_as_float(sr[c >> 5][c & 31]));
+                }
+                const float mx = mxr * sl2;
+                // keep the reference maximum unless it would let a weight exceed 2^8
+                if (mx > m_ref + 8.f) {
+                    corr = ex2(m_ref - mx);  // 0 on the first step
+                    m_ref = mx;
+                }
+                const float nmu = m_ref == -INFINITY ? 0.f : -m_ref;
+#pragma unroll
+                for (int c = 0; c < STEP; c += 2) {
+                    const float e0 = ex2(fmaf(__uint_as_float(sr[c >> 5][c & 31]), sl2, nmu));
+                    const float e1 =
+                        ex2(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), sl2, nmu));
+                    lsum += e0 + e1;
+                    pk[c >> 1] = pack_bf16x2(e0, e1);
+                }
+            } else {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < STEP; ++c) {
+                    float v = __uint_as_float(sr[c >> 5][c & 31]) * sl2;
+                    v = (t0 + c <= pos) ? v : -INFINITY;
+                    sr[c >> 5][c & 31] = __float_as_uint(v);
+                    mx = fmaxf(mx, v);
+                }
+                if (mx > m_ref + 8.f) {
+                    corr = ex2(m_ref - mx);
+                    m_ref = mx;
+                }
+                const float mu = m_ref == -INFINITY ? 0.f : m_ref;
+#pragma unroll
+                for (int c = 0; c < STEP; c += 2) {
+                    const float e0 = ex2(__uint_as_float(sr[c >> 5][c & 31]) - mu);
+                    const float e1 = ex2(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]) - mu);
+                    lsum += e0 + e1;
+                    pk[c >> 1] = pack_bf16x2(e0, e1);
+                }
             }
             l = l * corr + lsum;
 
