@@ -346,6 +346,7 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
 
     // every wait is bounded; a wait that gives up raises the abort flag and everyone leaves
     auto wait = [&](int b_idx, uint32_t parity) -> bool {
+        if (mbar_try_wait(bar(b_idx), parity)) return true;
         if (misc[1]) return false;
         if (mbar_wait_bounded(bar(b_idx), parity, WAIT_LIMIT_NS)) return true;
         misc[1] = 1;
@@ -462,35 +463,40 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             float corr = 1.f, lsum = 0.f;
             if (sl2 > 0.f) {
                 // fast path: maximum on the raw scores, one FMA + one EX2 per element
-                float mxr = -INFINITY;
+                float m8[8];  // eight independent chains, then a tree
+#pragma unroll
+                for (int i = 0; i < 8; ++i) m8[i] = -INFINITY;
                 if (__any_sync(0xffffffffu, t0 + STEP - 1 > pos)) {  // diagonal step: mask
 #pragma unroll
                     for (int c = 0; c < STEP; ++c) {
                         float v = __uint_as_float(sr[c >> 5][c & 31]);
                         v = (t0 + c <= pos) ? v : -INFINITY;
                         sr[c >> 5][c & 31] = __float_as_uint(v);
-                        mxr = fmaxf(mxr, v);
+                        m8[c & 7] = fmaxf(m8[c & 7], v);
                     }
                 } else {
 #pragma unroll
                     for (int c = 0; c < STEP; ++c)
-                        mxr = fmaxf(mxr, __uint_as_float(sr[c >> 5][c & 31]));
+                        m8[c & 7] = fmaxf(m8[c & 7], __uint_as_float(sr[c >> 5][c & 31]));
                 }
-                const float mx = mxr * sl2;
+                const float mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])),
+                                       fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7]))) * sl2;
                 // keep the reference maximum unless it would let a weight exceed 2^8
                 if (mx > m_ref + 8.f) {
                     corr = ex2(m_ref - mx);  // 0 on the first step
                     m_ref = mx;
                 }
                 const float nmu = m_ref == -INFINITY ? 0.f : -m_ref;
+                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c = 0; c < STEP; c += 2) {
                     const float e0 = ex2(fmaf(__uint_as_float(sr[c >> 5][c & 31]), sl2, nmu));
                     const float e1 =
                         ex2(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), sl2, nmu));
-                    lsum += e0 + e1;
+                    ls4[(c >> 1) & 3] += e0 + e1;
                     pk[c >> 1] = pack_bf16x2(e0, e1);
                 }
+                lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
             } else {
                 float mx = -INFINITY;
 #pragma unroll
@@ -515,11 +521,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             }
             l = l * corr + lsum;
 
-            // the P buffer of step j-2 must have been consumed
-            if (j >= 2) {
-                ok = wait(B_PVDONE + (j & 1), ((j >> 1) - 1) & 1);
-                if (!ok) break;
-            }
+            // The P buffer of step j-2 is free: the commit behind s_full(j) covers every MMA the
+            // issuer had queued before Q K^T of step j, and P V of step j-2 is one of them.
             // rescale O (only after the first step, and only once P V of step j-1 is complete)
             if (j >= 1 && __any_sync(0xffffffffu, corr != 1.f)) {
                 ok = wait(B_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
