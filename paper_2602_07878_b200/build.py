@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libpagedkv.so")
-SOURCES = ["common.cu", "pa_decode.cu", "kv_swap.cu", "kv_append.cu", "pa_prefill.cu"]
+SOURCES = ["common.cu", "pa_decode.cu", "kv_swap.cu", "kv_append.cu", "pa_prefill.cu", "sched_sim.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--use_fast_math", "-Xcompiler", "-fPIC", "-Xptxas", "-v",
@@ -21,6 +21,7 @@ def _stale() -> bool:
     t = os.path.getmtime(LIB)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps.append(os.path.join(_HERE, "..", "include", "pagedkv.h"))
+    deps.append(os.path.join(_HERE, "..", "include", "pagedkv_sched.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 

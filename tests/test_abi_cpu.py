@@ -18,15 +18,19 @@ def L():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "pagedkv.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"^\s*(?:const\s+char\s*\*|int64_t|int)\s+(\w+)\s*\(", text, flags=re.M)
+    names = []
+    for header in ("pagedkv.h", "pagedkv_sched.h"):
+        text = open(os.path.join(ROOT, "include", header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names += re.findall(r"^\s*(?:const\s+char\s*\*|void\s*\*|int64_t|int|void)\s+(\w+)\s*\(",
+                            text, flags=re.M)
     return names
 
 
 def test_header_symbols_are_exported(L):
     names = declared_functions()
-    assert {"pa_decode", "kv_swap_out", "kv_swap_in", "pa_workspace_bytes"} <= set(names)
+    assert {"pa_decode", "kv_swap_out", "kv_swap_in", "pa_workspace_bytes", "pa_prefill",
+            "kv_append", "sched_create", "sched_step", "sched_destroy"} <= set(names)
     for n in names:
         assert hasattr(L, n), f"{n} declared in pagedkv.h but not exported"
     assert set(api.EXPORTS) <= set(names)
