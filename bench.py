@@ -398,7 +398,7 @@ def run_ours(args):
     if rank == 0 and world == 1:
         line["kv_append"] = bench_append(torch, api, spec, k, v)
         if not args.no_recompute:
-            line["recompute"] = bench_recompute(torch, api, spec, k, v, tables)
+            line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -721,6 +721,8 @@ def main():
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-recompute", action="store_true")
+    ap.add_argument("--recompute-chunk", type=int, default=512,
+                    help="query tokens per pa_prefill call of the recompute leg")
     ap.add_argument("--cpu-fraction", type=float, default=1.0,
                     help="fraction of the batch's tokens the CPU baseline pass covers")
     ap.add_argument("--swap-pool-blocks", type=int, default=6144)
