@@ -29,6 +29,10 @@ def run_and_check(spec, partition_tokens=0, what=""):
 def test_cfg1_tiny_mha_matches_oracle():
     rel, g, out, ref = run_and_check(wl.config_spec(1))
     assert rel < 1e-2        # bf16 output rounding is ~2^-9 of the row maximum
+    # the same comparison against the stored oracle values (tests/golden)
+    from test_golden_cpu import load_golden
+    for b, h, d, x in load_golden():
+        assert abs(out[b, h, d] - x) <= 1e-2
 
 
 @pytest.mark.parametrize("P", [16, 32, 64, 128, 512])
