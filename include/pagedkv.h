@@ -275,6 +275,16 @@ int kv_swap_in(const kv_pool_desc* pool, const pa_shape* shape, void* k_pool, vo
 int pa_profile_enable(int on);
 int pa_profile_read(double* plan_ms, double* attention_ms, double* combine_ms, int64_t* calls);
 
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Every wait inside the
+ * kernels (on TMA data, on tensor-core completion, on another warp) gives up after a wall-
+ * clock limit, reports PA_STATUS_TIMEOUT and lets the kernel return, so that a lost signal
+ * costs an error code and not a hung GPU.  This call launches one warp that performs such a
+ * wait on a barrier nobody completes, with a limit of `limit_us` microseconds (1..100000),
+ * and ORs PA_STATUS_TIMEOUT into *dev_status (dev int32) when the limit has passed.
+ */
+int pa_selftest_wait_expiry(int32_t limit_us, int32_t* dev_status, void* cuda_stream);
+
 /* Text for a PA_* return code. */
 const char* pa_status_string(int code);
 

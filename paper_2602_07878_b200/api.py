@@ -31,7 +31,7 @@ EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_hos
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
            "pa_decode_static", "kv_append",
-           "pa_prefill_workspace_bytes", "pa_prefill"]
+           "pa_prefill_workspace_bytes", "pa_prefill", "pa_selftest_wait_expiry"]
 
 
 class PaShape(ctypes.Structure):
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.pa_prefill.argtypes = [pshape, vp, vp, vp, vp, i32, vp, vp, i32, i32, ctypes.c_float, vp,
                                  vp, sz, vp, vp]
         L.pa_prefill.restype = ctypes.c_int
+        L.pa_selftest_wait_expiry.argtypes = [i32, vp, vp]
+        L.pa_selftest_wait_expiry.restype = ctypes.c_int
         L.kv_append.argtypes = [pshape, vp, vp, vp, vp, vp, i32, vp, vp]
         L.kv_append.restype = ctypes.c_int
         L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
@@ -296,3 +298,9 @@ def pa_prefill(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, ou
                           _ptr(dev_status), _stream(stream))
     _check(rc, "pa_prefill")
     return out
+
+
+def pa_selftest_wait_expiry(limit_us: int, dev_status, stream=None):
+    """Forward to pa_selftest_wait_expiry: a bounded wait that must run out and report it."""
+    _check(lib().pa_selftest_wait_expiry(int(limit_us), _ptr(dev_status), _stream(stream)),
+           "pa_selftest_wait_expiry")

@@ -3,6 +3,7 @@
 #include <mutex>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace pk {
 
@@ -59,6 +60,31 @@ int validate_shape(const pa_shape* s) {
 }
 
 }  // namespace pk
+
+namespace pk {
+// One warp waits, with the same bounded wait the attention kernels use, on a barrier that
+// nobody will ever complete.  When the limit passes it reports PA_STATUS_TIMEOUT and returns.
+__global__ void wait_expiry_kernel(unsigned long long limit_ns, int* status) {
+    __shared__ __align__(8) unsigned long long barrier_word;
+    const uint32_t bar = smem_u32(&barrier_word);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        mbar_init_fence();
+    }
+    __syncwarp();
+    if (!mbar_wait_bounded(bar, 0, limit_ns) && threadIdx.x == 0)
+        atomicOr(status, PA_STATUS_TIMEOUT);
+}
+}  // namespace pk
+
+extern "C" int pa_selftest_wait_expiry(int32_t limit_us, int32_t* dev_status, void* cuda_stream) {
+    if (!dev_status) return PA_ERR_NULL;
+    if (limit_us <= 0 || limit_us > 100000) return PA_ERR_ARG;  // at most 0.1 s
+    pk::wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        (unsigned long long)limit_us * 1000ull, dev_status);
+    pk::count_launch();
+    return pk::check_cuda(cudaGetLastError());
+}
 
 extern "C" const char* pa_status_string(int code) {
     switch (code) {

@@ -207,3 +207,37 @@ def test_pa_decode_host_matches_device_call():
     api.pa_decode_host(qh, g.k, g.v, th, lh, spec.scale, oh, io, g.ws)
     torch.cuda.synchronize()
     assert torch.equal(oh.view(torch.int16), dev_out.view(torch.int16))
+
+
+def test_pa_decode_host_reads_large_tables_in_place():
+    # [32, 2048] int32 tables are 256 KiB: read in place over the host link, output posted in place
+    spec = wl.config_spec(3, scale_down=8)
+    q, k, v = small_inputs(spec)
+    g = GpuDecode(spec, q, k, v)
+    dev_out = g.run().cpu()
+    qh, th, lh = g.q.cpu().pin_memory(), g.tables.cpu().pin_memory(), g.lens.cpu().pin_memory()
+    assert th.numel() * 4 >= 256 << 10
+    oh = torch.zeros_like(qh).pin_memory()
+    shape = api.shape_of(g.k, spec.num_q_heads)
+    io = torch.empty(api.pa_host_io_bytes(shape, spec.batch, th.shape[1]), dtype=torch.uint8,
+                     device="cuda")
+    for _ in range(2):
+        api.pa_decode_host(qh, g.k, g.v, th, lh, spec.scale, oh, io, g.ws, dev_status=g.status)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int16), dev_out.view(torch.int16))
+    assert int(g.status.item()) == 0
+
+
+def test_a_wait_that_nobody_completes_times_out_and_reports_it():
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    api.pa_selftest_wait_expiry(2000, status)            # 2 ms limit
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == api.PA_STATUS_TIMEOUT
+    assert 1.5 < e0.elapsed_time(e1) < 100.0             # gave up after the limit, not much later
+    # the context is still usable
+    spec = wl.config_spec(1)
+    q, k, v = small_inputs(spec)
+    assert_parity(torch_to_f64(GpuDecode(spec, q, k, v).run()), oracle_for(spec, q, k, v))
