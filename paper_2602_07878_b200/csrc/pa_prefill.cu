@@ -269,19 +269,29 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 // O += P V (M 128, N 128, K 64).  Score buffers, P buffers and four KV stages are
 // double/quad buffered so that Q K^T of step j+1 overlaps the softmax of step j.
 namespace tc {
-constexpr int ROWS = 128, STEP = 64, ST = 4, D = 128;
+constexpr int ROWS = 128, STEP = 64, D = 128;
 constexpr int Q_BYTES = ROWS * D * 2;                 // two 64-dim halves of 128 rows x 128 B
 constexpr int KV_HALF = STEP * 128;                   // 64 tokens x 128 B
 constexpr int STAGE_BYTES = 4 * KV_HALF;              // K half 0, K half 1, V half 0, V half 1
 constexpr int P_BYTES = ROWS * STEP * 2;              // 128 rows x 64 tokens bf16
-constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + ST * STAGE_BYTES;
-constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
-// barriers (8 bytes each)
-enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + ST, B_SFULL = B_KVEMPTY + ST,
-       B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2, B_COUNT = B_PVDONE + 2 };
-constexpr int OFF_MISC = OFF_BAR + B_COUNT * 8;       // tmem base, abort flag, bad flag
-constexpr int SMEM_BYTES = OFF_MISC + 64 + 1024;      // + slack for 1024-byte alignment
-constexpr int TMEM_COLS = 256;                        // S0 [0,64) S1 [64,128) O [128,256)
+// NT = row tiles per CTA.  One tile: four KV stages and two P buffers.  Two tiles (two softmax
+// warpgroups taking turns on the tensor pipe) share three KV stages and have one P buffer each.
+template <int NT>
+struct Cfg {
+    static constexpr int ST = NT == 1 ? 4 : 3;
+    static constexpr int NP = NT == 1 ? 2 : 1;
+    static constexpr int OFF_Q = 0, OFF_KV = NT * Q_BYTES, OFF_P = OFF_KV + ST * STAGE_BYTES;
+    static constexpr int OFF_BAR = OFF_P + NT * NP * P_BYTES;
+    // barriers (8 bytes each): shared ones, then eight per tile
+    static constexpr int B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + ST, B_TILE = B_KVEMPTY + ST;
+    static constexpr int B_COUNT = B_TILE + 8 * NT;
+    static constexpr int OFF_MISC = OFF_BAR + B_COUNT * 8;  // tmem base, abort flag, bad flag
+    static constexpr int SMEM_BYTES = OFF_MISC + 64 + 1024;  // + slack for 1024-byte alignment
+    static constexpr int TMEM_COLS = 256 * NT;  // per tile: S0 [0,64) S1 [64,128) O [128,256)
+    static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + 1, THREADS = (4 * NT + 2) * 32;
+};
+// per-tile barrier indices, relative to Cfg::B_TILE + 8 * tile
+enum { T_SFULL = 0, T_SFREE = 2, T_PFULL = 4, T_PVDONE = 6 };
 }  // namespace tc
 
 struct PrefillTcParams {
@@ -289,11 +299,16 @@ struct PrefillTcParams {
     int tokens_per_tile;  // 128 / G
 };
 
-__global__ void __launch_bounds__(192, 1)
+template <int NT>
+__global__ void __launch_bounds__(tc::Cfg<NT>::THREADS, 1)
 pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                      const __grid_constant__ CUtensorMap kmap,
                      const __grid_constant__ CUtensorMap vmap, const PrefillTcParams tp) {
     using namespace tc;
+    using C = Cfg<NT>;
+    constexpr int ST = C::ST, NP = C::NP, OFF_Q = C::OFF_Q, OFF_KV = C::OFF_KV, OFF_P = C::OFF_P;
+    constexpr int OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC, TMEM_COLS = C::TMEM_COLS;
+    constexpr int B_QFULL = C::B_QFULL, B_KVFULL = C::B_KVFULL, B_KVEMPTY = C::B_KVEMPTY;
     const PrefillParams& p = tp.base;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -319,26 +334,27 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     }
     const int b = lo;
     const int q0 = p.cu_q_lens[b], ql = p.cu_q_lens[b + 1] - q0, L = p.ctx_lens[b];
-    const int tok0 = (gi - p.gstart[b]) * tpt;
-    const int ntok = min(tpt, ql - tok0);
-    const int pos_max = L - ql + tok0 + ntok - 1;
+    const int tok0 = (gi - p.gstart[b]) * (NT * tpt);   // first query token of the CTA
+    const int ntok_cta = min(NT * tpt, ql - tok0);
+    const int pos_max = L - ql + tok0 + ntok_cta - 1;
     const int n_steps = pos_max / STEP + 1;
     const int nblk_seq = (L + BS - 1) / BS;
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
         for (int i = 0; i < ST; ++i) mbar_init(bar(B_KVFULL + i), 1), mbar_init(bar(B_KVEMPTY + i), 1);
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(B_SFULL + i), 1);
-            mbar_init(bar(B_SFREE + i), 4);
-            mbar_init(bar(B_PFULL + i), 4);
-            mbar_init(bar(B_PVDONE + i), 1);
-        }
+        for (int t = 0; t < NT; ++t)
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(bar(C::B_TILE + 8 * t + T_SFULL + i), 1);
+                mbar_init(bar(C::B_TILE + 8 * t + T_SFREE + i), 4);
+                mbar_init(bar(C::B_TILE + 8 * t + T_PFULL + i), 4);
+                mbar_init(bar(C::B_TILE + 8 * t + T_PVDONE + i), 1);
+            }
         mbar_init_fence();
         misc[1] = 0;
         misc[2] = 0;
     }
-    if (warp == 5) tmem_alloc(sbase + OFF_MISC, TMEM_COLS);
+    if (warp == C::MMA_WARP) tmem_alloc(sbase + OFF_MISC, TMEM_COLS);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -354,15 +370,18 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         return false;
     };
 
-    if (warp == 4) {
+    if (warp == C::PRODUCER_WARP) {
         // ===================== TMA producer =====================
         if (lane == 0) {
             tma_prefetch_desc(&qmap);
             tma_prefetch_desc(&kmap);
             tma_prefetch_desc(&vmap);
-            mbar_arrive_expect_tx(bar(B_QFULL), Q_BYTES);
-            tma_load_4d(sbase + OFF_Q, &qmap, bar(B_QFULL), 0, 0, kvh, q0 + tok0);
-            tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &qmap, bar(B_QFULL), 64, 0, kvh, q0 + tok0);
+            mbar_arrive_expect_tx(bar(B_QFULL), NT * Q_BYTES);
+            for (int t = 0; t < NT; ++t) {  // tile t holds query tokens tok0 + t * tpt ..
+                const uint32_t qd = sbase + OFF_Q + t * Q_BYTES;
+                tma_load_4d(qd, &qmap, bar(B_QFULL), 0, 0, kvh, q0 + tok0 + t * tpt);
+                tma_load_4d(qd + Q_BYTES / 2, &qmap, bar(B_QFULL), 64, 0, kvh, q0 + tok0 + t * tpt);
+            }
         }
         const int32_t* table = p.block_tables + (size_t)b * p.max_blocks;
         int ids = lane < nblk_seq ? __ldg(&table[lane]) : p.NB;
@@ -393,70 +412,86 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                             0, kvh, used ? id : p.NB);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == C::MMA_WARP) {
         // ===================== MMA issuer (one thread) =====================
+        // Per step j: Q K^T of step j for every tile, then P V of step j-1 for every tile, so
+        // that the tensor pipe always has the other tile's work while one tile is in softmax.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = tc_idesc_bf16(ROWS, STEP, false);
             constexpr uint32_t idesc_pv = tc_idesc_bf16(ROWS, D, true);
             bool ok = wait(B_QFULL, 0);
             for (int j = 0; ok && j <= n_steps; ++j) {
-                if (j < n_steps) {  // S[j % 2] = Q K_j^T
+                if (j < n_steps) {  // S[tile][j % 2] = Q_tile K_j^T
                     const int stage = j % ST;
                     ok = wait(B_KVFULL + stage, (j / ST) & 1);
-                    if (ok && j >= 2) ok = wait(B_SFREE + (j & 1), ((j >> 1) - 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
                     const uint32_t kb = sbase + OFF_KV + stage * STAGE_BYTES;
+                    for (int t = 0; ok && t < NT; ++t) {
+                        const int tb = C::B_TILE + 8 * t;
+                        if (j >= 2) ok = wait(tb + T_SFREE + (j & 1), ((j >> 1) - 1) & 1);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t qb = sbase + OFF_Q + t * Q_BYTES;
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint64_t a = tc_smem_desc(
-                            sbase + OFF_Q + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32, 16, 1024);
-                        const uint64_t bd =
-                            tc_smem_desc(kb + (ks >> 2) * KV_HALF + (ks & 3) * 32, 16, 1024);
-                        tc_mma_bf16(tmem + (j & 1) * STEP, a, bd, idesc_qk, ks > 0);
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const uint64_t a =
+                                tc_smem_desc(qb + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32, 16, 1024);
+                            const uint64_t bd =
+                                tc_smem_desc(kb + (ks >> 2) * KV_HALF + (ks & 3) * 32, 16, 1024);
+                            tc_mma_bf16(tmem + t * 256 + (j & 1) * STEP, a, bd, idesc_qk, ks > 0);
+                        }
+                        tc_commit(bar(tb + T_SFULL + (j & 1)));
                     }
-                    tc_commit(bar(B_SFULL + (j & 1)));
-                }
-                if (j >= 1) {  // O += P_{j-1} V_{j-1}
-                    const int i = j - 1, stage = i % ST;
-                    ok = wait(B_PFULL + (i & 1), (i >> 1) & 1);
                     if (!ok) break;
-                    tc_fence_after_sync();
+                }
+                if (j >= 1) {  // O[tile] += P_{j-1} V_{j-1}
+                    const int i = j - 1, stage = i % ST;
                     const uint32_t vb = sbase + OFF_KV + stage * STAGE_BYTES + 2 * KV_HALF;
-                    const uint32_t pb = sbase + OFF_P + (i & 1) * P_BYTES;
+                    for (int t = 0; ok && t < NT; ++t) {
+                        const int tb = C::B_TILE + 8 * t;
+                        ok = wait(tb + T_PFULL + (i & 1), (i >> 1) & 1);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t pb = sbase + OFF_P + (t * NP + (i % NP)) * P_BYTES;
 #pragma unroll
-                    for (int kk = 0; kk < STEP / 16; ++kk) {
-                        const uint64_t a = tc_smem_desc(pb + kk * 32, 16, 1024);
-                        // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
-                        const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
-                        tc_mma_bf16(tmem + 2 * STEP, a, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < STEP / 16; ++kk) {
+                            const uint64_t a = tc_smem_desc(pb + kk * 32, 16, 1024);
+                            // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
+                            const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
+                            tc_mma_bf16(tmem + t * 256 + 2 * STEP, a, bd, idesc_pv,
+                                        (i > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        tc_commit(bar(tb + T_PVDONE + (i & 1)));
                     }
-                    tc_commit(bar(B_KVEMPTY + stage));
-                    tc_commit(bar(B_PVDONE + (i & 1)));
+                    if (!ok) break;
+                    tc_commit(bar(B_KVEMPTY + stage));  // every tile's P V of this stage is queued
                 }
             }
         }
     } else {
         // ===================== softmax + epilogue: thread = row =====================
-        const int row = tid;
+        const int ti = warp >> 2;                       // row tile of this warpgroup
+        const int row = (warp & 3) * 32 + lane;
         const int tk = row / G, hd = row - tk * G;
-        const bool row_ok = tk < ntok;
-        const int pos = row_ok ? L - ql + tok0 + tk : 0x7fffffff;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const int qtok = tok0 + ti * tpt + tk;          // query token within the sequence's chunk
+        const bool row_ok = qtok < ql;
+        const int pos = row_ok ? L - ql + qtok : 0x7fffffff;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tcol = tmem + ti * 256;          // this tile's S0, S1, O columns
+        const int tb = C::B_TILE + 8 * ti;              // this tile's barriers
         const float sl2 = p.scale_log2;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n_steps; ++j) {
-            ok = wait(B_SFULL + (j & 1), (j >> 1) & 1);
+            ok = wait(tb + T_SFULL + (j & 1), (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
             uint32_t sr[2][32];
-            tmem_ld32(tmem + lane_base + (j & 1) * STEP, sr[0]);
-            tmem_ld32(tmem + lane_base + (j & 1) * STEP + 32, sr[1]);
+            tmem_ld32(tcol + lane_base + (j & 1) * STEP, sr[0]);
+            tmem_ld32(tcol + lane_base + (j & 1) * STEP + 32, sr[1]);
             tmem_wait_ld();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_SFREE + (j & 1)));
+            if (lane == 0) mbar_arrive(bar(tb + T_SFREE + (j & 1)));
 
             const int t0 = j * STEP;
             uint32_t pk[STEP / 2];
@@ -521,27 +556,34 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             }
             l = l * corr + lsum;
 
-            // The P buffer of step j-2 is free: the commit behind s_full(j) covers every MMA the
-            // issuer had queued before Q K^T of step j, and P V of step j-2 is one of them.
+            // P V of step j-2 is complete: the commit behind s_full(j) covers every MMA the issuer
+            // had queued before Q K^T of step j.  With one P buffer per tile P V of step j-1 must
+            // be complete as well before the buffer is overwritten.
+            bool waited_prev = false;
+            if (NP == 1 && j >= 1) {
+                ok = wait(tb + T_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
+                if (!ok) break;
+                waited_prev = true;
+            }
             // rescale O (only after the first step, and only once P V of step j-1 is complete)
             if (j >= 1 && __any_sync(0xffffffffu, corr != 1.f)) {
-                ok = wait(B_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
+                if (!waited_prev) ok = wait(tb + T_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
 #pragma unroll 1
                 for (int c = 0; c < D; c += 32) {
                     uint32_t o[32];
-                    tmem_ld32(tmem + lane_base + 2 * STEP + c, o);
+                    tmem_ld32(tcol + lane_base + 2 * STEP + c, o);
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
-                    tmem_st32(tmem + lane_base + 2 * STEP + c, o);
+                    tmem_st32(tcol + lane_base + 2 * STEP + c, o);
                 }
                 tmem_wait_st();
             }
             // P row -> shared memory, 128-byte swizzle (16-byte chunk c of row r at c ^ (r & 7))
             {
-                const uint32_t prow = sbase + OFF_P + (j & 1) * P_BYTES + row * 128;
+                const uint32_t prow = sbase + OFF_P + (ti * NP + (j % NP)) * P_BYTES + row * 128;
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
                     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(
@@ -551,13 +593,13 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                                  : "memory");
             }
             // slots past the end of the sequence may hold anything: zero their V rows
-            if (t0 + STEP > L) {
+            if (ti == 0 && t0 + STEP > L) {  // one warpgroup does it; P V of every tile follows its p_full
                 ok = wait(B_KVFULL + (j % ST), (j / ST) & 1);
                 if (!ok) break;
                 const int r0 = max(0, L - t0);                      // first unused row of the step
                 const int r1 = min(STEP, ((L + BS - 1) / BS) * BS - t0);  // end of the partial block
                 const uint32_t vb = sbase + OFF_KV + (j % ST) * STAGE_BYTES + 2 * KV_HALF;
-                for (int e = tid; e < (r1 - r0) * 16; e += 128) {
+                for (int e = row; e < (r1 - r0) * 16; e += 128) {
                     const int r = r0 + (e >> 4), c = e & 15;  // 16 chunks: 8 per half
                     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(
                                      vb + (c >> 3) * KV_HALF + r * 128 + (c & 7) * 16),
@@ -568,20 +610,20 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             fence_proxy_async_smem();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_PFULL + (j & 1)));
+            if (lane == 0) mbar_arrive(bar(tb + T_PFULL + (j & 1)));
         }
         // ---- epilogue: O / l -> bf16 rows ----
-        if (ok) ok = wait(B_PVDONE + ((n_steps - 1) & 1), ((n_steps - 1) >> 1) & 1);
+        if (ok) ok = wait(tb + T_PVDONE + ((n_steps - 1) & 1), ((n_steps - 1) >> 1) & 1);
         if (ok) {
             tc_fence_after_sync();
             const bool bad = misc[2] != 0;
             const float inv = bad ? 0.f : 1.f / l;
             __nv_bfloat16* dst =
-                p.out + ((size_t)(q0 + tok0 + tk) * H + (size_t)kvh * G + hd) * D;
+                p.out + ((size_t)(q0 + qtok) * H + (size_t)kvh * G + hd) * D;
 #pragma unroll 1
             for (int c = 0; c < D; c += 32) {
                 uint32_t o[32];
-                tmem_ld32(tmem + lane_base + 2 * STEP + c, o);
+                tmem_ld32(tcol + lane_base + 2 * STEP + c, o);
                 tmem_wait_ld();
                 if (row_ok) {
 #pragma unroll
@@ -600,7 +642,7 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     // ---- teardown: everyone meets, then the allocating warp returns the tensor memory ----
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == C::MMA_WARP) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
@@ -639,25 +681,27 @@ static int make_q_map(CUtensorMap* map, const void* q, int total_q, int Hkv, int
     return PA_OK;
 }
 
+template <int NT>
 static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
-                             const PrefillTcParams& tp, int max_tiles, const DeviceInfo& dev,
+                             const PrefillTcParams& tp, int max_ctas, const DeviceInfo& dev,
                              cudaStream_t st) {
+    using C = tc::Cfg<NT>;
     static int configured_dev = -1;
     static std::mutex mu;
     {
         std::lock_guard<std::mutex> lk(mu);
         if (configured_dev != dev.device) {
-            int rc = check_cuda(cudaFuncSetAttribute(pa_prefill_tc_kernel,
+            int rc = check_cuda(cudaFuncSetAttribute(pa_prefill_tc_kernel<NT>,
                                                      cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                     tc::SMEM_BYTES));
+                                                     C::SMEM_BYTES));
             if (rc) return rc;
             configured_dev = dev.device;
         }
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(max_tiles);
-    cfg.blockDim = dim3(192);
-    cfg.dynamicSmemBytes = tc::SMEM_BYTES;
+    cfg.gridDim = dim3(max_ctas);
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -665,7 +709,7 @@ static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     count_launch();
-    return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_tc_kernel, qm, km, vm, tp));
+    return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_tc_kernel<NT>, qm, km, vm, tp));
 }
 
 }  // namespace pk
@@ -724,7 +768,19 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
         return e && std::string(e) == "mma";
     }();
     const bool use_tc = !force_mma && shape->head_dim == 128 && (128 % G) == 0;
-    plan.tpg = use_tc ? 128 / G : 16 / G;
+    // two row tiles per CTA (two softmax warpgroups sharing the K/V stages) once there are
+    // enough tiles to still give every SM a CTA; otherwise one tile per CTA
+    static const int forced_tiles = [] {
+        const char* e = std::getenv("PAGEDKV_PREFILL_TILES");
+        return e ? std::atoi(e) : 0;
+    }();
+    int tiles_per_cta = 1;
+    if (use_tc) {
+        const int64_t tiles = ((int64_t)total_q / (128 / G) + batch) * shape->num_kv_heads;
+        tiles_per_cta = tiles >= 2LL * dev.sm_count ? 2 : 1;
+        if (forced_tiles == 1 || forced_tiles == 2) tiles_per_cta = forced_tiles;
+    }
+    plan.tpg = use_tc ? tiles_per_cta * (128 / G) : 16 / G;
     plan.hdr = hdr;
     plan.gstart = hdr + PF_WORDS;
     plan.status = dev_status ? dev_status : hdr + PF_STATUS;
@@ -756,9 +812,10 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
         if (rc) return rc;
         PrefillTcParams tp;
         tp.base = pp;
-        tp.tokens_per_tile = plan.tpg;
-        const int max_tiles = (total_q / plan.tpg + batch) * pp.Hkv;
-        return launch_prefill_tc(qm, km, vm, tp, max_tiles, dev, st);
+        tp.tokens_per_tile = 128 / G;
+        const int max_ctas = (total_q / plan.tpg + batch) * pp.Hkv;
+        return tiles_per_cta == 2 ? launch_prefill_tc<2>(qm, km, vm, tp, max_ctas, dev, st)
+                                  : launch_prefill_tc<1>(qm, km, vm, tp, max_ctas, dev, st);
     }
     return shape->head_dim == 128 ? launch_prefill<128>(km, vm, pp, dev, st)
                                   : launch_prefill<64>(km, vm, pp, dev, st);

@@ -120,3 +120,14 @@ def test_large_scores_and_growing_maxima():
     # the softmax is nearly one-hot here, so outputs are single V rows of magnitude 2-4 where
     # one bf16 step is 2^-6 = 0.0156: the absolute bound is widened to 2e-2 for this case only
     assert_parity(out, ref, "scale 8", abs_tol=2e-2)
+
+
+def test_large_chunk_takes_the_two_tile_kernel():
+    # (1300 / 32 + 2) * 8 KV heads = 336 tiles >= 2 x 148 SMs: two row tiles per CTA, two
+    # softmax warpgroups sharing the K/V stages; the second sequence ends in a half-used pair
+    spec, q, k, v, cu = make_case([1500, 777], [900, 400], 32, 8, 128, seed=60)
+    g = GpuPrefill(spec, q, k, v)
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, "two tiles per CTA")
