@@ -396,6 +396,7 @@ def run_ours(args):
     }
 
     if rank == 0 and world == 1:
+        line["probes"] = bench_probes(torch, api, peak, value / world, achieved)
         line["kv_append"] = bench_append(torch, api, spec, k, v)
         if not args.no_recompute:
             line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk)
@@ -408,6 +409,29 @@ def run_ours(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def bench_probes(torch, api, copy_peak, step_gbps, kernel_gbps, gib=2, reps=5):
+    """Practical read ceilings measured in the same run: a read-only stream and 4 KiB gathers
+    (one bulk copy per granule, as the attention kernel fetches its tiles) over a 2 GiB buffer."""
+    buf = torch.empty(gib << 30, dtype=torch.uint8, device="cuda")
+    buf.zero_()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = {"bytes": buf.numel(), "copy_peak_gbps": copy_peak, "nominal_gbps": 8000.0}
+    for name, scattered in (("read_stream_gbps", False), ("read_gather_4k_gbps", True)):
+        best = 0.0
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            api.pa_probe_read(buf, scattered, status)
+            e1.record()
+            e1.synchronize()
+            best = max(best, buf.numel() / e0.elapsed_time(e1) / 1e6)
+        out[name] = best
+    assert int(status.item()) == 0
+    out["attention_kernel_frac_of_gather"] = kernel_gbps / out["read_gather_4k_gbps"]
+    out["step_frac_of_gather"] = step_gbps / out["read_gather_4k_gbps"]
+    return out
 
 
 def bench_append(torch, api, spec, k, v, calls=200):

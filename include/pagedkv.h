@@ -276,6 +276,19 @@ int pa_profile_enable(int on);
 int pa_profile_read(double* plan_ms, double* attention_ms, double* combine_ms, int64_t* calls);
 
 /*
+ * Read-bandwidth probe (no counterpart in the paper; a measurement aid).  One kernel reads
+ * `bytes` (rounded down to 4 KiB granules) of `dev_buf` and nothing else: granule by granule
+ * in order (scattered = 0) or in a pseudo-random order that visits every granule once
+ * (scattered != 0), each granule with one bulk asynchronous copy into shared memory -- the
+ * mechanism and granule size of the attention kernel's K/V tiles.  bytes / elapsed time is the
+ * practical ceiling for a read-only stream, respectively for 4 KiB gathers out of a fragmented
+ * pool.  dev_sink (dev, 8 bytes, may be NULL) is never written in practice; dev_status gets
+ * PA_STATUS_TIMEOUT if a bounded wait gives up.
+ */
+int pa_probe_read(const void* dev_buf, size_t bytes, int32_t scattered, uint32_t seed,
+                  void* dev_sink, int32_t* dev_status, void* cuda_stream);
+
+/*
  * Self-test of the bounded waits (no counterpart in the paper).  Every wait inside the
  * kernels (on TMA data, on tensor-core completion, on another warp) gives up after a wall-
  * clock limit, reports PA_STATUS_TIMEOUT and lets the kernel return, so that a lost signal

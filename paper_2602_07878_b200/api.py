@@ -31,7 +31,7 @@ EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_hos
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
            "pa_decode_static", "kv_append",
-           "pa_prefill_workspace_bytes", "pa_prefill", "pa_selftest_wait_expiry"]
+           "pa_prefill_workspace_bytes", "pa_prefill", "pa_selftest_wait_expiry", "pa_probe_read"]
 
 
 class PaShape(ctypes.Structure):
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.pa_prefill.restype = ctypes.c_int
         L.pa_selftest_wait_expiry.argtypes = [i32, vp, vp]
         L.pa_selftest_wait_expiry.restype = ctypes.c_int
+        L.pa_probe_read.argtypes = [vp, sz, i32, ctypes.c_uint32, vp, vp, vp]
+        L.pa_probe_read.restype = ctypes.c_int
         L.kv_append.argtypes = [pshape, vp, vp, vp, vp, vp, i32, vp, vp]
         L.kv_append.restype = ctypes.c_int
         L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
@@ -304,3 +306,9 @@ def pa_selftest_wait_expiry(limit_us: int, dev_status, stream=None):
     """Forward to pa_selftest_wait_expiry: a bounded wait that must run out and report it."""
     _check(lib().pa_selftest_wait_expiry(int(limit_us), _ptr(dev_status), _stream(stream)),
            "pa_selftest_wait_expiry")
+
+
+def pa_probe_read(buf, scattered: bool, dev_status, seed: int = 1, stream=None):
+    """Forward to pa_probe_read: read every 4 KiB granule of `buf` once, in order or scattered."""
+    _check(lib().pa_probe_read(_ptr(buf), buf.numel() * buf.element_size(), 1 if scattered else 0,
+                               seed, None, _ptr(dev_status), _stream(stream)), "pa_probe_read")

@@ -241,3 +241,14 @@ def test_a_wait_that_nobody_completes_times_out_and_reports_it():
     spec = wl.config_spec(1)
     q, k, v = small_inputs(spec)
     assert_parity(torch_to_f64(GpuDecode(spec, q, k, v).run()), oracle_for(spec, q, k, v))
+
+
+def test_read_probes_run_and_report_no_timeout():
+    buf = torch.zeros(64 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n0 = api.pa_launch_count()
+    api.pa_probe_read(buf, False, status)
+    api.pa_probe_read(buf, True, status, seed=7)
+    api.pa_probe_read(buf[: 4096 * 3], True, status)      # fewer granules than warps
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and api.pa_launch_count() - n0 == 3
