@@ -292,13 +292,15 @@ def run_ours(args):
     lens = torch.from_numpy(spec.seq_lens).to(dev)
     out = torch.empty_like(q)
     shape = api.shape_of(k, spec.num_q_heads)
-    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, spec.total_tokens + 16 * spec.batch),
+    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, spec.total_tokens + 16 * spec.batch,
+                                             args.partition_tokens),
                      dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     step_bytes = spec.algorithmic_bytes()
 
     def step():
-        api.pa_decode(q, k, v, tables, lens, spec.scale, out, ws, dev_status=status)
+        api.pa_decode(q, k, v, tables, lens, spec.scale, out, ws, dev_status=status,
+                      partition_tokens=args.partition_tokens)
 
     warmup = max(args.warmup, 3)
     for _ in range(warmup):
@@ -343,7 +345,8 @@ def run_ours(args):
                      device=dev)
 
     def step_e2e():
-        api.pa_decode_host(qh, k, v, th, lh, spec.scale, oh, io, ws, dev_status=status)
+        api.pa_decode_host(qh, k, v, th, lh, spec.scale, oh, io, ws, dev_status=status,
+                           partition_tokens=args.partition_tokens)
 
     for _ in range(3):
         step_e2e()
@@ -742,6 +745,8 @@ def main():
                     help="decode workload (3 = full-pool mixed-length GQA, the headline; "
                          "4 = full-size swap churn, 126 GB pool, 1 GPU)")
     ap.add_argument("--churn-steps", type=int, default=3)
+    ap.add_argument("--partition-tokens", type=int, default=0,
+                    help="force the decode partition size (0 = chosen per call on the device)")
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-recompute", action="store_true")
