@@ -160,3 +160,37 @@ def test_full_size_swap_churn_and_decode():
     qh, kh, vh, tables, lens, ids = host_inputs_for(spec, sample, layer)
     ref = oracle.pa_decode(qh, kh, vh, tables, lens, spec.scale)
     assert_parity(torch_to_f64(out[sample]), ref, "workload 4 decode after churn")
+
+
+def test_decode_time_is_linear_in_total_context_once_bandwidth_bound():
+    """Eq. 3 of the paper models the attention step's time as context bytes / HBM bandwidth.
+    Doubling every context length must therefore about double the step's device time once
+    the batch is far larger than L2."""
+    times = {}
+    for mult in (1, 2, 4):
+        lens = np.full(96, 2048 * mult, np.int64)
+        spec = wl.make_spec("t", seq_lens=lens, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                            occupancy=0.97, seed=mult)
+        n = spec.num_blocks * spec.block_elems
+        shape = (spec.num_blocks, 8, 16, 128)
+        k = wl.normal_bf16_torch(0, n, 1, "cuda").view(shape)
+        v = wl.normal_bf16_torch(0, n, 2, "cuda").view(shape)
+        q = wl.q_torch(spec, "cuda")
+        tables = torch.from_numpy(spec.block_tables).cuda()
+        lens_d = torch.from_numpy(spec.seq_lens).cuda()
+        out = torch.empty_like(q)
+        ws = torch.empty(api.pa_workspace_bytes(api.shape_of(k, 32), 96, spec.total_tokens + 2048),
+                         dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            api.pa_decode(q, k, v, tables, lens_d, spec.scale, out, ws)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            api.pa_decode(q, k, v, tables, lens_d, spec.scale, out, ws)
+        e1.record()
+        e1.synchronize()
+        times[mult] = e0.elapsed_time(e1) / 20
+        assert spec.kv_bytes() > 4 * (126 << 20)
+        del k, v
+    assert 1.8 < times[2] / times[1] < 2.2, times
+    assert 1.8 < times[4] / times[2] < 2.2, times
