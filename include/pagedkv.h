@@ -106,7 +106,9 @@ int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch, int64_t max_tot
  *   seq_lens     dev int32 [batch]; 0 gives a row of zeros
  *   scale        softmax scale (e.g. 1/sqrt(D))
  *   out          dev bf16 [batch, H, D], contiguous, 16-byte aligned
- *   workspace    dev, >= pa_workspace_bytes(...), 256-byte aligned; contents are scratch
+ *   workspace    dev, >= pa_workspace_bytes(...), 256-byte aligned; contents are scratch.
+ *                One call at a time per workspace: calls that may overlap on the GPU (different
+ *                streams) need a workspace each
  *   partition_tokens  0 = choose per call from the batch's total length; otherwise a
  *                multiple of 16 in [16, 512]: sequences longer than this are split into
  *                partitions of this many tokens that run in parallel and are merged by

@@ -11,6 +11,8 @@ from paper_2602_07878_b200 import workloads as wl
 # per (sequence, head) row, max_d |gpu - ref| <= 2e-2 * max_d |ref|.
 ABS_TOL = 1e-2
 REL_TOL = 2e-2
+GUARD = 4096            # guard elements on each side of a test's output buffer
+GUARD_BITS = 0x7A5A     # their content (int16 view)
 
 
 def assert_parity(gpu: np.ndarray, ref: np.ndarray, what: str = "", abs_tol: float = ABS_TOL):
@@ -52,12 +54,20 @@ class GpuDecode:
             spec.block_tables if tables is None else tables)).to(dev)
         self.lens = torch.from_numpy(np.ascontiguousarray(
             spec.seq_lens if lens is None else lens).astype(np.int32)).to(dev)
-        self.out = torch.full_like(self.q, float("nan"))
+        # output and workspace sit between guard zones holding a bit pattern: with no memory
+        # checker available, a kernel that writes outside its buffers is caught here
+        n_out = self.q.numel()
+        self._out_store = torch.full((n_out + 2 * GUARD,), GUARD_BITS, dtype=torch.int16, device=dev)
+        self.out = self._out_store[GUARD:GUARD + n_out].view(torch.bfloat16).view(self.q.shape)
+        self.out.fill_(float("nan"))
         shape = api.shape_of(self.k, self.q.shape[1])
         tot = int(max_tokens if max_tokens is not None else
                   self.tables.shape[0] * self.tables.shape[1] * 16)
         nbytes = api.pa_workspace_bytes(shape, self.q.shape[0], tot, partition_tokens)
-        self.ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        nbytes = (nbytes + 255) & ~255
+        self._ws_store = torch.full((nbytes + 2 * 4096,), 0x5A, dtype=torch.uint8, device=dev)
+        self.ws = self._ws_store[4096:4096 + nbytes]
+        assert self.ws.data_ptr() % 256 == 0
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.partition_tokens = partition_tokens
 
@@ -68,7 +78,15 @@ class GpuDecode:
                       self.spec.scale if scale is None else scale, self.out, self.ws,
                       dev_status=self.status, **kw)
         torch.cuda.synchronize()
+        self.check_guards()
         return self.out
+
+    def check_guards(self):
+        n = self.q.numel()
+        assert bool((self._out_store[:GUARD] == GUARD_BITS).all()), "write before the output"
+        assert bool((self._out_store[GUARD + n:] == GUARD_BITS).all()), "write past the output"
+        assert bool((self._ws_store[:4096] == 0x5A).all()), "write before the workspace"
+        assert bool((self._ws_store[4096 + self.ws.numel():] == 0x5A).all()), "write past the workspace"
 
     def plan_header(self):
         return self.ws[:64 * 4].view(torch.int32).cpu().numpy()
