@@ -65,7 +65,7 @@ extern "C" {
 typedef struct pa_shape {
     int32_t num_q_heads;  /* H; a multiple of num_kv_heads, H / Hkv <= 16                  */
     int32_t num_kv_heads; /* Hkv                                                           */
-    int32_t head_dim;     /* D: 64 or 128                                                  */
+    int32_t head_dim;     /* D: 64, 128 or 256                                             */
     int32_t block_size;   /* tokens per block: 16                                          */
     int32_t num_blocks;   /* physical pool size                                            */
     int32_t dtype;        /* PA_BF16                                                       */

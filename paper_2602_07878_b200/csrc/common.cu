@@ -46,7 +46,7 @@ int get_device_info(DeviceInfo* info) {
 
 int validate_shape(const pa_shape* s) {
     if (s->dtype != PA_BF16) return PA_ERR_SHAPE;
-    if (s->head_dim != 64 && s->head_dim != 128) return PA_ERR_SHAPE;
+    if (s->head_dim != 64 && s->head_dim != 128 && s->head_dim != 256) return PA_ERR_SHAPE;
     if (s->block_size != BS) return PA_ERR_SHAPE;
     if (s->num_kv_heads <= 0 || s->num_q_heads <= 0) return PA_ERR_SHAPE;
     if (s->num_q_heads % s->num_kv_heads) return PA_ERR_SHAPE;

@@ -65,7 +65,7 @@ extern "C" int kv_append(const pa_shape* shape, void* k_cache, void* v_cache, co
     p.total_slots = (int64_t)shape->num_blocks * BS;
     p.batch = batch;
     p.Hkv = shape->num_kv_heads;
-    p.log2_vec = shape->head_dim == 128 ? 4 : 3;
+    p.log2_vec = shape->head_dim == 256 ? 5 : shape->head_dim == 128 ? 4 : 3;
     const int64_t threads = (int64_t)batch * p.Hkv << p.log2_vec;
     const unsigned grid = (unsigned)((threads + 255) / 256);
     kv_append_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);

@@ -117,7 +117,7 @@ static int swap_common(const SwapCall& c, bool out) {
     p.stride_head = s.stride_head * 2;
     p.stride_tok = s.stride_tok * 2;
     p.layers = c.pool->num_layers;
-    p.log2_d = s.head_dim == 128 ? 7 : 6;
+    p.log2_d = s.head_dim == 256 ? 8 : s.head_dim == 128 ? 7 : 6;
     p.vec_per_chunk = (int)(chunk_bytes / 16);
 
     for (int32_t done = 0; done < c.n; done += per_launch) {

@@ -484,9 +484,12 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) 
             const size_t r = (size_t)(first + min(i0 + 4 * u, np - 1)) * p.H + h;
             ml[u] = p.partial_ml[r];
             const float* src = p.partial_o + r * D + lane * VPL;
-            if (VPL == 4) {
-                const float4 x = *reinterpret_cast<const float4*>(src);
-                v[u][0] = x.x, v[u][1] = x.y, v[u][VPL - 2] = x.z, v[u][VPL - 1] = x.w;
+            if (VPL >= 4) {
+#pragma unroll
+                for (int i = 0; i + 3 < VPL; i += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(src + i);
+                    v[u][i] = x.x, v[u][i + 1] = x.y, v[u][i + 2] = x.z, v[u][i + 3] = x.w;
+                }
             } else {
                 const float2 x = *reinterpret_cast<const float2*>(src);
                 v[u][0] = x.x, v[u][1] = x.y;
@@ -514,11 +517,14 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) 
         const int c = lane * VPL + i;
         o[i] = ((s_acc[0][c] + s_acc[1][c]) + (s_acc[2][c] + s_acc[3][c])) * inv;
     }
-    if (VPL == 4) {
-        uint2 x;
-        x.x = bad ? 0u : pack_bf16x2(o[0], o[1]);
-        x.y = bad ? 0u : pack_bf16x2(o[VPL - 2], o[VPL - 1]);
-        *reinterpret_cast<uint2*>(dst + lane * VPL) = x;
+    if (VPL >= 4) {
+#pragma unroll
+        for (int i = 0; i + 3 < VPL; i += 4) {
+            uint2 x;
+            x.x = bad ? 0u : pack_bf16x2(o[i], o[i + 1]);
+            x.y = bad ? 0u : pack_bf16x2(o[i + 2], o[i + 3]);
+            *reinterpret_cast<uint2*>(dst + lane * VPL + i) = x;
+        }
     } else {
         *reinterpret_cast<uint32_t*>(dst + lane * VPL) = bad ? 0u : pack_bf16x2(o[0], o[1]);
     }
@@ -640,14 +646,19 @@ template <int D, bool HI>
 static int dispatch_variant(Variant v, const CUtensorMap& km, const CUtensorMap& vm,
                             const DecodeParams& dp, const DeviceInfo& dev, int* warps, bool launch,
                             cudaStream_t st) {
-    constexpr int F = 128 / D;  // a D=64 slot is half the size: twice the slots
+    if constexpr (D == 256) {
+        // a slot is 16 KiB: four warps with three slots each fill the shared memory
+        return launch_decode<D, HI, 4, 3>(km, vm, dp, dev, warps, launch, st);
+    } else {
+        constexpr int F = D == 64 ? 2 : 1;  // a D=64 slot is half the size: twice the slots
 #define PK_CASE(NW_, NS_) \
     if (v.nw == NW_ && v.nslot == NS_) \
         return launch_decode<D, HI, NW_, NS_ * F>(km, vm, dp, dev, warps, launch, st);
-    PK_CASE(8, 3)
-    PK_CASE(4, 3)
+        PK_CASE(8, 3)
+        PK_CASE(4, 3)
 #undef PK_CASE
-    return PA_ERR_ARG;
+        return PA_ERR_ARG;
+    }
 }
 
 static Variant chosen_variant() {
@@ -667,6 +678,9 @@ static int dispatch_decode(const pa_shape* s, const CUtensorMap& km, const CUten
                            cudaStream_t st) {
     const bool hi = s->num_q_heads / s->num_kv_heads > 8;
     const Variant v = chosen_variant();
+    if (s->head_dim == 256)
+        return hi ? dispatch_variant<256, true>(v, km, vm, dp, dev, warps, launch, st)
+                  : dispatch_variant<256, false>(v, km, vm, dp, dev, warps, launch, st);
     if (s->head_dim == 128)
         return hi ? dispatch_variant<128, true>(v, km, vm, dp, dev, warps, launch, st)
                   : dispatch_variant<128, false>(v, km, vm, dp, dev, warps, launch, st);
@@ -820,7 +834,8 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     cp.counter_reset = 3 * total_warps;
     const int cgrid = cp.rows;
     count_launch();
-    rc = check_cuda(D == 128 ? launch_pdl(pa_combine_kernel<128>, dim3(cgrid), dim3(128), 0, st, cp)
+    rc = check_cuda(D == 256 ? launch_pdl(pa_combine_kernel<256>, dim3(cgrid), dim3(128), 0, st, cp)
+                    : D == 128 ? launch_pdl(pa_combine_kernel<128>, dim3(cgrid), dim3(128), 0, st, cp)
                              : launch_pdl(pa_combine_kernel<64>, dim3(cgrid), dim3(128), 0, st, cp));
     if (prof) cudaEventRecord(prof_ev.ev[3], st);
     return rc;

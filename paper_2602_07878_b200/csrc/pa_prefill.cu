@@ -230,7 +230,7 @@ pa_prefill_kernel(const __grid_constant__ CUtensorMap kmap,
 template <int D>
 static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const PrefillParams& pp,
                           const DeviceInfo& dev, cudaStream_t st) {
-    constexpr int NW = 8, NSLOT = 3 * (128 / D);
+    constexpr int NW = D == 256 ? 4 : 8, NSLOT = D == 64 ? 6 : 3;
     auto kern = pa_prefill_kernel<D, NW, NSLOT>;
     const int smem = NW * NSLOT * (2 * BS * D * 2) + NW * NSLOT * 8 + 1024;
     static int configured_dev = -1;
@@ -817,6 +817,7 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
         return tiles_per_cta == 2 ? launch_prefill_tc<2>(qm, km, vm, tp, max_ctas, dev, st)
                                   : launch_prefill_tc<1>(qm, km, vm, tp, max_ctas, dev, st);
     }
-    return shape->head_dim == 128 ? launch_prefill<128>(km, vm, pp, dev, st)
-                                  : launch_prefill<64>(km, vm, pp, dev, st);
+    return shape->head_dim == 256   ? launch_prefill<256>(km, vm, pp, dev, st)
+           : shape->head_dim == 128 ? launch_prefill<128>(km, vm, pp, dev, st)
+                                    : launch_prefill<64>(km, vm, pp, dev, st);
 }

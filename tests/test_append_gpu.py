@@ -16,7 +16,7 @@ def as_bits(t):
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("Hkv,D", [(8, 128), (2, 64), (5, 128)])
+@pytest.mark.parametrize("Hkv,D", [(8, 128), (2, 64), (5, 128), (8, 256)])
 def test_append_bit_exact_and_nothing_else_changes(Hkv, D):
     lens = np.arange(0, 70, 3)
     spec = wl.make_spec("t", seq_lens=lens, num_q_heads=Hkv, num_kv_heads=Hkv, head_dim=D,

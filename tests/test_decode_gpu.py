@@ -42,7 +42,8 @@ def test_cfg1_forced_partitions(P):
 
 @pytest.mark.parametrize("H,Hkv,D", [(4, 4, 64), (8, 2, 64), (8, 2, 128), (32, 8, 128),
                                      (8, 1, 128), (16, 1, 128), (32, 2, 64), (6, 3, 128),
-                                     (12, 1, 64), (5, 5, 128)])
+                                     (12, 1, 64), (5, 5, 128), (16, 8, 256), (4, 4, 256),
+                                     (16, 1, 256), (6, 2, 256)])
 def test_head_layouts(H, Hkv, D):
     lens = [1, 15, 16, 17, 31, 33, 0, 70, 129, 513, 1000, 2049]
     spec = wl.make_spec("t", seq_lens=lens, num_q_heads=H, num_kv_heads=Hkv, head_dim=D,

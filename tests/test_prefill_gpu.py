@@ -43,7 +43,8 @@ def make_case(ctx, qlens, H, Hkv, D, seed):
 
 @pytest.mark.parametrize("H,Hkv,D", [(8, 8, 64), (8, 2, 128), (32, 8, 128), (16, 1, 128),
                                      (6, 2, 64), (10, 2, 128), (8, 1, 64), (4, 4, 128),
-                                     (8, 4, 128), (8, 1, 128), (64, 8, 128)])
+                                     (8, 4, 128), (8, 1, 128), (64, 8, 128), (16, 8, 256),
+                                     (4, 1, 256)])
 def test_mixed_chunks_match_oracle(H, Hkv, D):
     ctx = [37, 64, 5, 130, 1, 700, 16, 333]
     qlens = [37, 10, 0, 33, 1, 512, 16, 1]

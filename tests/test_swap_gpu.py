@@ -23,7 +23,7 @@ def as_bits(t):
 
 
 @pytest.mark.parametrize("staged", [False, True])
-@pytest.mark.parametrize("layers,NB,Hkv,D", [(1, 40, 8, 64), (3, 64, 2, 128), (32, 24, 8, 128)])
+@pytest.mark.parametrize("layers,NB,Hkv,D", [(1, 40, 8, 64), (3, 64, 2, 128), (32, 24, 8, 128), (2, 30, 8, 256)])
 def test_swap_out_and_in_bit_exact(staged, layers, NB, Hkv, D):
     k, v = make_pools(layers, NB, Hkv, D)
     kd, vd = bits_to_torch(k), bits_to_torch(v)
