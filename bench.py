@@ -414,6 +414,99 @@ def run_ours(args):
         print(json.dumps(line))
 
 
+def run_seqsplit(args):
+    """`--seq-split`: every context of the workload is split by blocks over the N ranks
+    (strong scaling: the job's KV bytes are fixed).  A step = partial attention over the
+    rank's slice, an all-gather of the partial records over NCCL, the merge.  Every rank
+    generates the whole synthetic pool and reads only its slice of it."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_07878_b200 import api, build as lib_build, seqsplit
+    from paper_2602_07878_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if "MASTER_ADDR" in os.environ:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29655", rank=0, world_size=1,
+                                device_id=torch.device("cuda", local))
+    if rank == 0:
+        lib_build.build()
+    dist.barrier()
+    dev = "cuda"
+    spec = wl.config_spec(args.workload)
+    q = wl.q_torch(spec, dev)
+    k, v = wl.pools_torch(spec, dev)
+    t_np, l_np = seqsplit.shard_context(spec.block_tables, spec.seq_lens, rank, world,
+                                        spec.block_size)
+    tables, lens = torch.from_numpy(t_np).to(dev), torch.from_numpy(l_np).to(dev)
+    out = torch.empty_like(q)
+    shape = api.shape_of(k, spec.num_q_heads)
+    local_tokens = int(l_np.sum())
+    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, local_tokens + 16 * spec.batch,
+                                            args.partition_tokens), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    n = api.pa_partial_floats(shape, spec.batch)
+    part = torch.empty(n, dtype=torch.float32, device=dev)
+    gathered = torch.empty((world, n), dtype=torch.float32, device=dev)
+
+    def step():
+        seqsplit.decode(q, k, v, tables, lens, spec.scale, out, ws, part, gathered,
+                        dev_status=status, partition_tokens=args.partition_tokens)
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    dist.barrier()
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = api.pa_launch_count()
+    with ClockSampler(local) as clocks:
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+    launches = api.pa_launch_count() - n0
+    dist.barrier()
+    # bytes this rank's kernels must move per step: its slice of the KV, q, its table entries,
+    # its record out, all records in, the output rows
+    kv_local = local_tokens * 2 * spec.num_kv_heads * spec.head_dim * 2
+    rank_bytes = (kv_local + q.numel() * 2 + int(((l_np + 15) // 16).sum()) * 4 + spec.batch * 4
+                  + n * 4 * (1 + world) + out.numel() * 2)
+    ms, total_bytes = aggregate_over_ranks(e0.elapsed_time(e1), float(rank_bytes) * args.steps, dist)
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    peak, peak_src = measured_peaks()
+    value = total_bytes / ms / 1e6
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "num_q_heads": spec.num_q_heads,
+                   "num_kv_heads": spec.num_kv_heads, "head_dim": spec.head_dim,
+                   "total_context_tokens": spec.total_tokens,
+                   "parallelism": f"sequence split over {world} rank(s): partial attention, "
+                                  "all-gather of partial records (NCCL), merge",
+                   "exchange_bytes_per_rank_per_step": n * 4,
+                   "l2": "inputs (KV read per step) exceed the 126 MB L2 at N=1; no flush"},
+        "tokens_per_s": spec.batch * args.steps / (ms / 1e3),
+        "frac_of_hbm_peak": value / world / peak, "peak_source": peak_src,
+        "gpu_launches": int(launches), "clocks": clocks.summary(),
+    }
+    dist.barrier()
+    dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
 def bench_probes(torch, api, copy_peak, step_gbps, kernel_gbps, gib=2, reps=5):
     """Practical read ceilings measured in the same run: a read-only stream and 4 KiB gathers
     (one bulk copy per granule, as the attention kernel fetches its tiles) over a 2 GiB buffer."""
@@ -747,6 +840,9 @@ def main():
     ap.add_argument("--churn-steps", type=int, default=3)
     ap.add_argument("--partition-tokens", type=int, default=0,
                     help="force the decode partition size (0 = chosen per call on the device)")
+    ap.add_argument("--seq-split", action="store_true",
+                    help="split every context over the ranks (one all-gather per step) "
+                         "instead of running independent replicas")
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-recompute", action="store_true")
@@ -764,6 +860,8 @@ def main():
         run_reference(args)
     elif args.workload == 4:
         run_churn(args)
+    elif args.seq_split:
+        run_seqsplit(args)
     else:
         run_ours(args)
 

@@ -164,6 +164,41 @@ int pa_decode_static(const pa_shape* shape, const void* q, const void* k_cache,
                      int64_t max_total_tokens, float scale, void* out, int32_t partition_tokens,
                      int32_t* dev_status, void* cuda_stream);
 
+/* ---- sequence-split decode: one context sharded over several GPUs -------------------------
+ * Tensor-parallel serving (Section 6.4, TP 2/4/8) shards KV heads, which needs no exchange
+ * inside this path.  A context can also be split by tokens: each rank keeps a slice of every
+ * sequence's blocks, attends over its slice, and the ranks exchange one small record per
+ * rank before a final merge.  The merge is the same log-sum-exp combine that joins the
+ * partitions of one call.
+ *
+ * A partial record for `rows` = batch * num_q_heads output rows of width D is
+ * rows * (D + 2) floats: first the un-normalised accumulators o[rows][D]
+ * (o = sum_t 2^(s_t - m) V_t over the rank's tokens, s_t = scale * log2(e) * <q, K_t>), then
+ * (m, l)[rows] pairs with m the maximum of s_t and l = sum_t 2^(s_t - m).  A row whose
+ * slice is empty has o = 0, m = -inf, l = 0; a row that met a bad block id has m = NaN.
+ *
+ * pa_partial_floats: floats to set aside for one record: rows * (D + 2) rounded up to a
+ *   multiple of 4, so that records packed back to back stay 16-byte aligned.
+ * pa_decode_partial: pa_decode over the rank's slice (its own block table rows and local
+ *   lengths), result written as one record to `part` (device, 16-byte aligned).  All other
+ *   arguments, the workspace and the errors are those of pa_decode.
+ * pa_merge_partials: out[row] = sum_i 2^(m_i - M) o_i[row] / sum_i 2^(m_i - M) l_i, M = max m_i,
+ *   rounded to bf16; a row with l = 0 in every record, or NaN in any, is zeros.  `parts` is a
+ *   HOST array of num_parts (<= PA_MAX_PARTS) DEVICE pointers, each to one record; they are
+ *   copied before return.  The kernel reads them with plain loads only, so a pointer may
+ *   be a peer GPU's memory mapped into this process; the caller orders the merge after the
+ *   records are complete (an all-gather on the same stream, or an event / barrier across
+ *   ranks for peer pointers).  out: device bf16 [rows][head_dim]. */
+#define PA_MAX_PARTS 32
+int pa_partial_floats(const pa_shape* shape, int32_t batch, size_t* floats);
+int pa_decode_partial(const pa_shape* shape, const void* q, const void* k_cache,
+                      const void* v_cache, const int32_t* block_tables,
+                      int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
+                      float scale, float* part, void* workspace, size_t workspace_bytes,
+                      int32_t partition_tokens, int32_t* dev_status, void* cuda_stream);
+int pa_merge_partials(const float* const* parts, int32_t num_parts, int32_t rows,
+                      int32_t head_dim, void* out, void* cuda_stream);
+
 /* Bytes of device buffer pa_decode_host needs for its device copies of q, block tables,
  * lengths and out. */
 int pa_host_io_bytes(const pa_shape* shape, int32_t max_batch, int32_t max_blocks_per_seq,

@@ -30,7 +30,8 @@ PA_STATIC_WORKSPACE_BYTES = 64 << 20
 EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
-           "pa_decode_static", "kv_append",
+           "pa_decode_static", "kv_append", "pa_partial_floats", "pa_decode_partial",
+           "pa_merge_partials",
            "pa_prefill_workspace_bytes", "pa_prefill", "pa_selftest_wait_expiry", "pa_probe_read"]
 
 
@@ -75,6 +76,13 @@ def lib() -> ctypes.CDLL:
         L.pa_decode_static.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, i64, ctypes.c_float,
                                        vp, i32, vp, vp]
         L.pa_decode_static.restype = ctypes.c_int
+        L.pa_partial_floats.argtypes = [pshape, i32, psz]
+        L.pa_partial_floats.restype = ctypes.c_int
+        L.pa_decode_partial.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp,
+                                        vp, sz, i32, vp, vp]
+        L.pa_decode_partial.restype = ctypes.c_int
+        L.pa_merge_partials.argtypes = [ctypes.POINTER(vp), i32, i32, i32, vp, vp]
+        L.pa_merge_partials.restype = ctypes.c_int
         L.pa_prefill_workspace_bytes.argtypes = [i32, psz]
         L.pa_prefill_workspace_bytes.restype = ctypes.c_int
         L.pa_prefill.argtypes = [pshape, vp, vp, vp, vp, i32, vp, vp, i32, i32, ctypes.c_float, vp,
@@ -156,6 +164,52 @@ def pa_decode(q, k_cache, v_cache, block_tables, seq_lens, scale, out, workspace
                          workspace.numel() * workspace.element_size(), partition_tokens, flags,
                          _ptr(dev_status), _stream(stream))
     _check(rc, "pa_decode")
+    return out
+
+
+def pa_partial_floats(shape: PaShape, batch: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().pa_partial_floats(ctypes.byref(shape), batch, ctypes.byref(out)),
+           "pa_partial_floats")
+    return int(out.value)
+
+
+def pa_decode_partial(q, k_cache, v_cache, block_tables, seq_lens, scale, part, workspace, *,
+                      partition_tokens: int = 0, dev_status=None, stream=None,
+                      shape: Optional[PaShape] = None):
+    """Forward to pa_decode_partial: attention over this rank's slice of every sequence,
+    written to `part` (float32, B*H*(D+2) elements) as one partial record."""
+    if shape is None:
+        shape = shape_of(k_cache, q.shape[1])
+        assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
+    assert block_tables.dtype == torch.int32 and seq_lens.dtype == torch.int32
+    assert q.is_contiguous() and block_tables.is_contiguous()
+    assert part.dtype == torch.float32 and part.is_contiguous()
+    assert part.numel() >= q.shape[0] * q.shape[1] * (q.shape[2] + 2)
+    rc = lib().pa_decode_partial(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                 _ptr(block_tables),
+                                 block_tables.shape[1] if block_tables.dim() == 2 else 0,
+                                 _ptr(seq_lens), q.shape[0], float(scale), _ptr(part),
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                 partition_tokens, _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_decode_partial")
+    return part
+
+
+def pa_merge_partials(parts, rows: int, head_dim: int, out, stream=None):
+    """Forward to pa_merge_partials.  `parts`: a list of float32 tensors (one record each), or
+    one [R, rows*(D+2)] tensor as an all-gather leaves it; out bf16 [rows, D] (any shape with
+    that many contiguous elements)."""
+    if isinstance(parts, torch.Tensor):
+        assert parts.dim() == 2 and parts.is_contiguous()
+        parts = [parts[i] for i in range(parts.shape[0])]
+    for t in parts:
+        assert t.dtype == torch.float32 and t.is_contiguous()
+        assert t.numel() >= rows * (head_dim + 2)
+    assert out.dtype == torch.bfloat16 and out.is_contiguous() and out.numel() == rows * head_dim
+    arr = (ctypes.c_void_p * max(1, len(parts)))(*[t.data_ptr() for t in parts])
+    rc = lib().pa_merge_partials(arr, len(parts), rows, head_dim, _ptr(out), _stream(stream))
+    _check(rc, "pa_merge_partials")
     return out
 
 

@@ -38,6 +38,7 @@ struct PlanParams {
     int max_blocks;
     int Hkv;
     int forced_p;       // 0 = automatic
+    int no_direct;      // 1 = every sequence goes through the combine kernel
     int64_t item_cap;   // records the workspace can hold
     int total_warps;    // decode warps on the chip
     int* hdr;
@@ -188,7 +189,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
             const int ntok = min(P, L - tok0);
             const int nb = (ntok + BS - 1) / BS;
             const int pos = start[nb] + atomicAdd(&cursor[nb], 1);
-            p.records[pos] = make_int4(b, tok0, ntok | (np == 1 ? REC_DIRECT : 0), first + part);
+            p.records[pos] =
+                make_int4(b, tok0, ntok | (np == 1 && !p.no_direct ? REC_DIRECT : 0), first + part);
         }
     }
 }
@@ -436,13 +438,21 @@ struct CombineParams {
     int rows;  // batch * H
     int H;
     int counter_reset;
+    // COMBINE_TO_PARTIAL: one un-normalised fp32 row and its (max, sum) per output row
+    float* part_o;
+    float2* part_ml;
+    // COMBINE_MERGE: the partitions of row r are row r of each of n_parts records
+    int n_parts;
+    const float* parts[PA_MAX_PARTS];
 };
+
+enum { COMBINE_FINAL = 0, COMBINE_TO_PARTIAL = 1, COMBINE_MERGE = 2 };
 
 // One CTA (4 warps) per (sequence, query head) row.  Every warp finds the row maximum, then
 // the warps share the partitions (warp w takes w, w+4, ...), eight independent 512-byte row
 // loads at a time, and the four partial sums meet in shared memory.
-template <int D>
-__global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) {
+template <int D, int MODE>
+__global__ void __launch_bounds__(128) pa_combine_kernel(const __grid_constant__ CombineParams p) {
     constexpr int VPL = D / 32;  // floats per lane
     constexpr int UB = 8;        // rows in flight per warp
     __shared__ float s_acc[4][D];
@@ -451,20 +461,37 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     pdl_wait();  // partial results of the attention kernel are complete and visible
-    if (row == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
+    if (MODE != COMBINE_MERGE && row == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
     const int b = row / p.H, h = row - b * p.H;
-    const int2 info = p.seq_info[b];
-    if (info.y == 1) return;  // written directly by the attention kernel
+    const int2 info = MODE == COMBINE_MERGE ? make_int2(0, p.n_parts) : p.seq_info[b];
+    if (MODE == COMBINE_FINAL && info.y == 1) return;  // written directly by the attention kernel
     __nv_bfloat16* dst = p.out + (size_t)row * D;
-    if (info.y == 0) {  // no tokens: a row of zeros
-        if (threadIdx.x < D / 2) reinterpret_cast<uint32_t*>(dst)[threadIdx.x] = 0u;
+    if (info.y == 0) {  // no tokens: a row of zeros (as a partial: weight zero)
+        if (MODE == COMBINE_TO_PARTIAL) {
+            if (threadIdx.x < D / 2)
+                reinterpret_cast<float2*>(p.part_o + (size_t)row * D)[threadIdx.x] =
+                    make_float2(0.f, 0.f);
+            if (threadIdx.x == 0) p.part_ml[row] = make_float2(-INFINITY, 0.f);
+        } else if (threadIdx.x < D / 2) {
+            reinterpret_cast<uint32_t*>(dst)[threadIdx.x] = 0u;
+        }
         return;
     }
     const int np = info.y, first = info.x;
+    // partition i of this row: its (max, sum) pair and its accumulator row
+    auto ml_of = [&](int i) -> float2 {
+        if (MODE == COMBINE_MERGE)
+            return reinterpret_cast<const float2*>(p.parts[i] + (size_t)p.rows * D)[row];
+        return p.partial_ml[(size_t)(first + i) * p.H + h];
+    };
+    auto o_of = [&](int i) -> const float* {
+        if (MODE == COMBINE_MERGE) return p.parts[i] + (size_t)row * D;
+        return p.partial_o + ((size_t)(first + i) * p.H + h) * D;
+    };
     float M = -INFINITY;
     bool bad = false;
     for (int i = lane; i < np; i += 32) {
-        const float m = p.partial_ml[(size_t)(first + i) * p.H + h].x;
+        const float m = ml_of(i).x;
         bad |= m != m;  // NaN marks a partition that met a bad block id
         M = fmaxf(M, m);
     }
@@ -481,9 +508,9 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) 
         float v[UB][VPL];
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
-            const size_t r = (size_t)(first + min(i0 + 4 * u, np - 1)) * p.H + h;
-            ml[u] = p.partial_ml[r];
-            const float* src = p.partial_o + r * D + lane * VPL;
+            const int idx = min(i0 + 4 * u, np - 1);
+            ml[u] = ml_of(idx);
+            const float* src = o_of(idx) + lane * VPL;
             if (VPL >= 4) {
 #pragma unroll
                 for (int i = 0; i + 3 < VPL; i += 4) {
@@ -510,12 +537,22 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const CombineParams p) 
     __syncthreads();
     if (warp != 0) return;
     den = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
-    const float inv = bad ? 0.f : 1.f / den;
+    // a row without any token in every part (den == 0) is a row of zeros
+    const float inv = MODE == COMBINE_TO_PARTIAL ? 1.f : (bad || den == 0.f) ? 0.f : 1.f / den;
     float o[VPL];
 #pragma unroll
     for (int i = 0; i < VPL; ++i) {
         const int c = lane * VPL + i;
         o[i] = ((s_acc[0][c] + s_acc[1][c]) + (s_acc[2][c] + s_acc[3][c])) * inv;
+    }
+    if (MODE == COMBINE_TO_PARTIAL) {
+        float* po = p.part_o + (size_t)row * D + lane * VPL;
+#pragma unroll
+        for (int i = 0; i < VPL; i += 2)
+            *reinterpret_cast<float2*>(po + i) = make_float2(o[i], o[i + 1]);
+        if (lane == 0)
+            p.part_ml[row] = make_float2(bad ? __int_as_float(0x7fc00000) : M, den);
+        return;
     }
     if (VPL >= 4) {
 #pragma unroll
@@ -737,12 +774,21 @@ extern "C" int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch,
     return PA_OK;
 }
 
-extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cache,
-                         const void* v_cache, const int32_t* block_tables,
-                         int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
-                         float scale, void* out, void* workspace, size_t workspace_bytes,
-                         int32_t partition_tokens, int32_t flags, int32_t* dev_status,
-                         void* cuda_stream) {
+template <int MODE>
+static cudaError_t launch_combine(int D, int grid, cudaStream_t st, const CombineParams& cp) {
+    return D == 256   ? launch_pdl(pa_combine_kernel<256, MODE>, dim3(grid), dim3(128), 0, st, cp)
+           : D == 128 ? launch_pdl(pa_combine_kernel<128, MODE>, dim3(grid), dim3(128), 0, st, cp)
+                      : launch_pdl(pa_combine_kernel<64, MODE>, dim3(grid), dim3(128), 0, st, cp);
+}
+
+// The three launches of a decode call.  `part` == nullptr: bf16 rows in `out`; otherwise one
+// partial record (un-normalised fp32 rows, then their (max, sum) pairs) in `part`.
+static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache,
+                       const void* v_cache, const int32_t* block_tables,
+                       int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
+                       float scale, void* out, float* part, void* workspace,
+                       size_t workspace_bytes, int32_t partition_tokens, int32_t flags,
+                       int32_t* dev_status, void* cuda_stream) {
     if (!shape) return PA_ERR_NULL;
     int rc = validate_shape(shape);
     if (rc) return rc;
@@ -752,10 +798,11 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
         return PA_ERR_ARG;
     if (flags & ~PA_FLAG_REUSE_PLAN) return PA_ERR_ARG;
     if (batch == 0) return PA_OK;
-    if (!q || !k_cache || !v_cache || !block_tables || !seq_lens || !out || !workspace)
+    if (!q || !k_cache || !v_cache || !block_tables || !seq_lens || !(part ? (void*)part : out) ||
+        !workspace)
         return PA_ERR_NULL;
-    if (!aligned16(q) || !aligned16(out) || !aligned16(k_cache) || !aligned16(v_cache) ||
-        (reinterpret_cast<uintptr_t>(workspace) & 255))
+    if (!aligned16(q) || !aligned16(part ? (void*)part : out) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || (reinterpret_cast<uintptr_t>(workspace) & 255))
         return PA_ERR_ALIGN;
     if ((int64_t)max_blocks_per_seq * BS > INT32_MAX) return PA_ERR_ARG;
 
@@ -807,6 +854,7 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
         pp.max_blocks = max_blocks_per_seq;
         pp.Hkv = shape->num_kv_heads;
         pp.forced_p = partition_tokens;
+        pp.no_direct = part != nullptr;
         pp.item_cap = w.item_cap;
         pp.total_warps = total_warps;
         pp.hdr = hdr;
@@ -823,7 +871,7 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     if (rc) return rc;
     if (prof) cudaEventRecord(prof_ev.ev[2], st);
 
-    CombineParams cp;
+    CombineParams cp = {};
     cp.seq_info = reinterpret_cast<const int2*>(ws + w.off_seqinfo);
     cp.partial_o = dp.partial_o;
     cp.partial_ml = dp.partial_ml;
@@ -832,13 +880,73 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     cp.rows = batch * H;
     cp.H = H;
     cp.counter_reset = 3 * total_warps;
+    if (part) {
+        cp.part_o = part;
+        cp.part_ml = reinterpret_cast<float2*>(part + (size_t)cp.rows * D);
+    }
     const int cgrid = cp.rows;
     count_launch();
-    rc = check_cuda(D == 256 ? launch_pdl(pa_combine_kernel<256>, dim3(cgrid), dim3(128), 0, st, cp)
-                    : D == 128 ? launch_pdl(pa_combine_kernel<128>, dim3(cgrid), dim3(128), 0, st, cp)
-                             : launch_pdl(pa_combine_kernel<64>, dim3(cgrid), dim3(128), 0, st, cp));
+    rc = check_cuda(part ? launch_combine<COMBINE_TO_PARTIAL>(D, cgrid, st, cp)
+                         : launch_combine<COMBINE_FINAL>(D, cgrid, st, cp));
     if (prof) cudaEventRecord(prof_ev.ev[3], st);
     return rc;
+}
+
+extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cache,
+                         const void* v_cache, const int32_t* block_tables,
+                         int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
+                         float scale, void* out, void* workspace, size_t workspace_bytes,
+                         int32_t partition_tokens, int32_t flags, int32_t* dev_status,
+                         void* cuda_stream) {
+    return decode_impl(shape, q, k_cache, v_cache, block_tables, max_blocks_per_seq, seq_lens,
+                       batch, scale, out, nullptr, workspace, workspace_bytes, partition_tokens,
+                       flags, dev_status, cuda_stream);
+}
+
+extern "C" int pa_partial_floats(const pa_shape* shape, int32_t batch, size_t* floats) {
+    if (!shape || !floats) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (batch < 0) return PA_ERR_ARG;
+    const size_t n = (size_t)batch * shape->num_q_heads * (shape->head_dim + 2);
+    *floats = (n + 3) & ~(size_t)3;  // records packed back to back stay 16-byte aligned
+    return PA_OK;
+}
+
+extern "C" int pa_decode_partial(const pa_shape* shape, const void* q, const void* k_cache,
+                                 const void* v_cache, const int32_t* block_tables,
+                                 int32_t max_blocks_per_seq, const int32_t* seq_lens,
+                                 int32_t batch, float scale, float* part, void* workspace,
+                                 size_t workspace_bytes, int32_t partition_tokens,
+                                 int32_t* dev_status, void* cuda_stream) {
+    if (batch > 0 && !part) return PA_ERR_NULL;
+    return decode_impl(shape, q, k_cache, v_cache, block_tables, max_blocks_per_seq, seq_lens,
+                       batch, scale, nullptr, part, workspace, workspace_bytes, partition_tokens,
+                       0, dev_status, cuda_stream);
+}
+
+extern "C" int pa_merge_partials(const float* const* parts, int32_t num_parts, int32_t rows,
+                                 int32_t head_dim, void* out, void* cuda_stream) {
+    if (num_parts < 0 || num_parts > PA_MAX_PARTS || rows < 0) return PA_ERR_ARG;
+    if (head_dim != 64 && head_dim != 128 && head_dim != 256) return PA_ERR_SHAPE;
+    if (rows == 0) return PA_OK;
+    if (!out || (num_parts > 0 && !parts)) return PA_ERR_NULL;
+    if (!aligned16(out)) return PA_ERR_ALIGN;
+    CombineParams cp = {};
+    for (int i = 0; i < num_parts; ++i) {
+        if (!parts[i]) return PA_ERR_NULL;
+        if (!aligned16(parts[i])) return PA_ERR_ALIGN;
+        cp.parts[i] = parts[i];
+    }
+    cp.out = static_cast<__nv_bfloat16*>(out);
+    cp.rows = rows;
+    cp.H = 1;
+    cp.n_parts = num_parts;
+    DeviceInfo dev;
+    int rc = get_device_info(&dev);
+    if (rc) return rc;
+    count_launch();
+    return check_cuda(launch_combine<COMBINE_MERGE>(head_dim, rows, static_cast<cudaStream_t>(cuda_stream), cp));
 }
 
 extern "C" int pa_profile_enable(int on) {
