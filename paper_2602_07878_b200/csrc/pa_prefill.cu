@@ -264,34 +264,35 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 // ======================================================================================
 // Warps 0-3: softmax and epilogue (thread i owns row i = TMEM lane i); warp 4: TMA producer;
 // warp 5: MMA issuer.  Per 64-token KV step:  S = Q K^T (M 128, N 64, K 128) into one of two
-// TMEM score buffers, the softmax warps turn S into bf16 weights P in shared memory (and
-// rescale the TMEM accumulator O when a row maximum has grown by more than 2^8), then
-// O += P V (M 128, N 128, K 64).  Score buffers, P buffers and four KV stages are
-// double/quad buffered so that Q K^T of step j+1 overlaps the softmax of step j.
+// TMEM score buffers, the softmax warps turn S into bf16 weights P written back over the
+// first 32 columns of that score buffer (and rescale the TMEM accumulator O when a row
+// maximum has grown by more than 2^8), then O += P V (M 128, N 128, K 64) with P read from
+// tensor memory: the weights never touch shared memory, whose bandwidth the two MMAs'
+// operand reads already fill.  Two score buffers and four KV stages let Q K^T of step j+1
+// overlap the softmax of step j.
 namespace tc {
 constexpr int ROWS = 128, STEP = 64, D = 128;
 constexpr int Q_BYTES = ROWS * D * 2;                 // two 64-dim halves of 128 rows x 128 B
 constexpr int KV_HALF = STEP * 128;                   // 64 tokens x 128 B
 constexpr int STAGE_BYTES = 4 * KV_HALF;              // K half 0, K half 1, V half 0, V half 1
-constexpr int P_BYTES = ROWS * STEP * 2;              // 128 rows x 64 tokens bf16
-// NT = row tiles per CTA.  One tile: four KV stages and two P buffers.  Two tiles (two softmax
-// warpgroups taking turns on the tensor pipe) share three KV stages and have one P buffer each.
+// NT = row tiles per CTA (two tiles = two softmax warpgroups taking turns on the tensor pipe
+// and sharing the KV stages).
 template <int NT>
 struct Cfg {
-    static constexpr int ST = NT == 1 ? 4 : 3;
-    static constexpr int NP = NT == 1 ? 2 : 1;
-    static constexpr int OFF_Q = 0, OFF_KV = NT * Q_BYTES, OFF_P = OFF_KV + ST * STAGE_BYTES;
-    static constexpr int OFF_BAR = OFF_P + NT * NP * P_BYTES;
+    static constexpr int ST = 4;
+    static constexpr int OFF_Q = 0, OFF_KV = NT * Q_BYTES;
+    static constexpr int OFF_BAR = OFF_KV + ST * STAGE_BYTES;
     // barriers (8 bytes each): shared ones, then eight per tile
     static constexpr int B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + ST, B_TILE = B_KVEMPTY + ST;
     static constexpr int B_COUNT = B_TILE + 8 * NT;
     static constexpr int OFF_MISC = OFF_BAR + B_COUNT * 8;  // tmem base, abort flag, bad flag
     static constexpr int SMEM_BYTES = OFF_MISC + 64 + 1024;  // + slack for 1024-byte alignment
-    static constexpr int TMEM_COLS = 256 * NT;  // per tile: S0 [0,64) S1 [64,128) O [128,256)
+    // per tile: S0 [0,64) S1 [64,128) O [128,256); P of step j lies over S(j % 2) [0,32)
+    static constexpr int TMEM_COLS = 256 * NT;
     static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + 1, THREADS = (4 * NT + 2) * 32;
 };
 // per-tile barrier indices, relative to Cfg::B_TILE + 8 * tile
-enum { T_SFULL = 0, T_SFREE = 2, T_PFULL = 4, T_PVDONE = 6 };
+enum { T_SFULL = 0, T_PFULL = 2, T_PVDONE = 4 };
 }  // namespace tc
 
 struct PrefillTcParams {
@@ -306,7 +307,7 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                      const __grid_constant__ CUtensorMap vmap, const PrefillTcParams tp) {
     using namespace tc;
     using C = Cfg<NT>;
-    constexpr int ST = C::ST, NP = C::NP, OFF_Q = C::OFF_Q, OFF_KV = C::OFF_KV, OFF_P = C::OFF_P;
+    constexpr int ST = C::ST, OFF_Q = C::OFF_Q, OFF_KV = C::OFF_KV;
     constexpr int OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC, TMEM_COLS = C::TMEM_COLS;
     constexpr int B_QFULL = C::B_QFULL, B_KVFULL = C::B_KVFULL, B_KVEMPTY = C::B_KVEMPTY;
     const PrefillParams& p = tp.base;
@@ -346,7 +347,6 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         for (int t = 0; t < NT; ++t)
             for (int i = 0; i < 2; ++i) {
                 mbar_init(bar(C::B_TILE + 8 * t + T_SFULL + i), 1);
-                mbar_init(bar(C::B_TILE + 8 * t + T_SFREE + i), 4);
                 mbar_init(bar(C::B_TILE + 8 * t + T_PFULL + i), 4);
                 mbar_init(bar(C::B_TILE + 8 * t + T_PVDONE + i), 1);
             }
@@ -416,6 +416,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         // ===================== MMA issuer (one thread) =====================
         // Per step j: Q K^T of step j for every tile, then P V of step j-1 for every tile, so
         // that the tensor pipe always has the other tile's work while one tile is in softmax.
+        // S(j % 2) is free for Q K^T of step j once P V of step j-2, which read its weights
+        // from there, has been issued: MMAs of one thread execute in issue order.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = tc_idesc_bf16(ROWS, STEP, false);
             constexpr uint32_t idesc_pv = tc_idesc_bf16(ROWS, D, true);
@@ -427,9 +429,6 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                     const uint32_t kb = sbase + OFF_KV + stage * STAGE_BYTES;
                     for (int t = 0; ok && t < NT; ++t) {
                         const int tb = C::B_TILE + 8 * t;
-                        if (j >= 2) ok = wait(tb + T_SFREE + (j & 1), ((j >> 1) - 1) & 1);
-                        if (!ok) break;
-                        tc_fence_after_sync();
                         const uint32_t qb = sbase + OFF_Q + t * Q_BYTES;
 #pragma unroll
                         for (int ks = 0; ks < D / 16; ++ks) {
@@ -451,14 +450,13 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                         ok = wait(tb + T_PFULL + (i & 1), (i >> 1) & 1);
                         if (!ok) break;
                         tc_fence_after_sync();
-                        const uint32_t pb = sbase + OFF_P + (t * NP + (i % NP)) * P_BYTES;
+                        const uint32_t pt = tmem + t * 256 + (i & 1) * STEP;
 #pragma unroll
                         for (int kk = 0; kk < STEP / 16; ++kk) {
-                            const uint64_t a = tc_smem_desc(pb + kk * 32, 16, 1024);
                             // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
                             const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
-                            tc_mma_bf16(tmem + t * 256 + 2 * STEP, a, bd, idesc_pv,
-                                        (i > 0 || kk > 0) ? 1u : 0u);
+                            tc_mma_bf16_ta(tmem + t * 256 + 2 * STEP, pt + kk * 8, bd, idesc_pv,
+                                           (i > 0 || kk > 0) ? 1u : 0u);
                         }
                         tc_commit(bar(tb + T_PVDONE + (i & 1)));
                     }
@@ -489,9 +487,6 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             tmem_ld32(tcol + lane_base + (j & 1) * STEP, sr[0]);
             tmem_ld32(tcol + lane_base + (j & 1) * STEP + 32, sr[1]);
             tmem_wait_ld();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(tb + T_SFREE + (j & 1)));
 
             const int t0 = j * STEP;
             uint32_t pk[STEP / 2];
@@ -556,18 +551,9 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             }
             l = l * corr + lsum;
 
-            // P V of step j-2 is complete: the commit behind s_full(j) covers every MMA the issuer
-            // had queued before Q K^T of step j.  With one P buffer per tile P V of step j-1 must
-            // be complete as well before the buffer is overwritten.
-            bool waited_prev = false;
-            if (NP == 1 && j >= 1) {
-                ok = wait(tb + T_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
-                if (!ok) break;
-                waited_prev = true;
-            }
             // rescale O (only after the first step, and only once P V of step j-1 is complete)
             if (j >= 1 && __any_sync(0xffffffffu, corr != 1.f)) {
-                if (!waited_prev) ok = wait(tb + T_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
+                ok = wait(tb + T_PVDONE + ((j - 1) & 1), ((j - 1) >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
 #pragma unroll 1
@@ -581,17 +567,9 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                 }
                 tmem_wait_st();
             }
-            // P row -> shared memory, 128-byte swizzle (16-byte chunk c of row r at c ^ (r & 7))
-            {
-                const uint32_t prow = sbase + OFF_P + (ti * NP + (j % NP)) * P_BYTES + row * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(
-                                     prow + ((c ^ (row & 7)) << 4)),
-                                 "r"(pk[4 * c]), "r"(pk[4 * c + 1]), "r"(pk[4 * c + 2]),
-                                 "r"(pk[4 * c + 3])
-                                 : "memory");
-            }
+            // P row -> tensor memory, over the scores just read: 64 bf16 in 32 columns
+            tmem_st32(tcol + lane_base + (j & 1) * STEP, pk);
+            bool zeroed = false;
             // slots past the end of the sequence may hold anything: zero their V rows
             if (ti == 0 && t0 + STEP > L) {  // one warpgroup does it; P V of every tile follows its p_full
                 ok = wait(B_KVFULL + (j % ST), (j / ST) & 1);
@@ -606,8 +584,10 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                                  "r"(0u)
                                  : "memory");
                 }
+                zeroed = true;
             }
-            fence_proxy_async_smem();
+            if (zeroed) fence_proxy_async_smem();
+            tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(tb + T_PFULL + (j & 1)));
