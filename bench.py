@@ -402,7 +402,8 @@ def run_ours(args):
         line["probes"] = bench_probes(torch, api, peak, value / world, achieved)
         line["kv_append"] = bench_append(torch, api, spec, k, v)
         if not args.no_recompute:
-            line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk)
+            line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk,
+                                                args.recompute_split)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -558,28 +559,35 @@ def bench_append(torch, api, spec, k, v, calls=200):
             "gbps": nbytes / us / 1e3, "bound": "launch latency / host issue rate (2 MB moved per call)"}
 
 
-def bench_recompute(torch, api, spec, k, v, tables, chunk=512):
+def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_splits=16):
     """Recomputation recovery of the longest sequence of the batch: causal prefill attention
-    over its cached tokens in chunks of `chunk` query tokens (one pa_prefill call per chunk,
-    context growing).  A dense contraction: reported in TFLOP/s against the bf16 tensor peak."""
+    over its cached tokens in chunks of `chunk` query tokens (one pa_prefill_split call per
+    chunk, context growing, the block table passed no wider than the context).  A dense
+    contraction: reported in TFLOP/s against the bf16 tensor peak."""
     b = int(np.argmax(spec.seq_lens))
     L = int(spec.seq_lens[b])
     H, D = spec.num_q_heads, spec.head_dim
     q = torch.empty(L, H, D, dtype=torch.bfloat16, device="cuda").normal_()
     out = torch.empty_like(q)
     tab = tables[b:b + 1].contiguous()
-    ws = torch.empty(api.pa_prefill_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(api.pa_prefill_split_workspace_bytes(api.shape_of(k, H), 1, min(chunk, L),
+                                                          max_splits),
+                     dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     calls = []
     for start in range(0, L, chunk):
         end = min(L, start + chunk)
         calls.append((start, end, torch.tensor([end], dtype=torch.int32, device="cuda"),
-                      torch.tensor([0, end - start], dtype=torch.int32, device="cuda")))
+                      torch.tensor([0, end - start], dtype=torch.int32, device="cuda"),
+                      tab[:, :(end + 15) // 16].contiguous()))
+    shapes = []
 
     def run():
-        for start, end, ctx, cu in calls:
-            api.pa_prefill(q[start:end], k, v, tab, ctx, cu, spec.scale, out[start:end], ws,
-                           dev_status=status)
+        shapes.clear()
+        for start, end, ctx, cu, t in calls:
+            api.pa_prefill_split(q[start:end], k, v, t, ctx, cu, spec.scale, out[start:end], ws,
+                                 kv_split_tokens=split, dev_status=status)
+            shapes.append(api.pa_prefill_last_launch())
 
     run()
     torch.cuda.synchronize()
@@ -590,7 +598,7 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512):
     e1.synchronize()
     ms = e0.elapsed_time(e1)
     # 4 * D flops per (query, visible key, head): QK^T and PV, 2 flops per multiply-add
-    pairs = sum((end - start) * (start + end + 1) // 2 for start, end, _, _ in calls)
+    pairs = sum((end - start) * (start + end + 1) // 2 for start, end, _, _, _ in calls)
     flops = 4.0 * D * H * pairs
     peak = None
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -599,6 +607,8 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512):
             peak = float(json.load(f)["bf16_tflops"])
     assert int(status.item()) == 0
     return {"tokens": L, "chunk": chunk, "calls": len(calls), "ms": ms, "tflops": flops / ms / 1e9,
+            "last_call_launch": {"tiles_per_cta": shapes[-1][0], "kv_split_tokens": shapes[-1][1],
+                                 "kv_splits": shapes[-1][2]},
             "bound": "tensor", "peak_tflops": peak,
             "frac": (flops / ms / 1e9 / peak) if peak else None,
             "tokens_per_s": L / (ms / 1e3)}
@@ -848,6 +858,8 @@ def main():
     ap.add_argument("--no-recompute", action="store_true")
     ap.add_argument("--recompute-chunk", type=int, default=512,
                     help="query tokens per pa_prefill call of the recompute leg")
+    ap.add_argument("--recompute-split", type=int, default=0,
+                    help="kv_split_tokens of the recompute leg (0 = library's choice, -1 = never)")
     ap.add_argument("--cpu-fraction", type=float, default=1.0,
                     help="fraction of the batch's tokens the CPU baseline pass covers")
     ap.add_argument("--swap-pool-blocks", type=int, default=6144)

@@ -250,6 +250,41 @@ int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const 
                void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
+ * pa_prefill with the KV range of a tile split over several CTAs (flash-decoding applied to
+ * the recomputation chunk of Section 5.1.2 / Appendix B.1: a 512-token chunk of one long
+ * victim yields fewer 128-row tiles than the GPU has SMs, while each tile walks tens of
+ * thousands of cached tokens).  The result is the same function of the inputs as pa_prefill;
+ * only the order of the fp32 sums differs.  A sequence whose context spans more than one
+ * split leaves per-split partial rows in the workspace, merged by a third kernel.
+ *
+ *   kv_split_tokens   0: the library chooses tile shape and split length from the chunk
+ *                     size, max_blocks_per_seq (taken as the bound of every context: pass
+ *                     a table no wider than the contexts need) and what the workspace holds;
+ *                     > 0: split length in tokens (rounded up to a multiple of 64);
+ *                     PA_ERR_WORKSPACE if ceil(max_blocks_per_seq * 16 / split) partial
+ *                     rows per query row do not fit; < 0: never split.
+ *   workspace         dev, 256-byte aligned, >= pa_prefill_workspace_bytes(batch); splits are
+ *                     used up to what pa_prefill_split_workspace_bytes(shape, batch, total_q,
+ *                     splits) says fits.
+ * Splitting needs head_dim 128 and a group size H / Hkv that divides 128 (the tensor-core
+ * kernel); other shapes run unsplit.  pa_prefill is this call with kv_split_tokens = 0.
+ * Two or three kernels are enqueued.  Errors as for pa_prefill; a split that met a bad
+ * block id zeroes the rows that depend on it.
+ */
+int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t max_batch,
+                                     int32_t max_total_q, int32_t max_splits, size_t* bytes);
+int pa_prefill_split(const pa_shape* shape, const void* q, const void* k_cache,
+                     const void* v_cache, const int32_t* block_tables,
+                     int32_t max_blocks_per_seq, const int32_t* ctx_lens,
+                     const int32_t* cu_q_lens, int32_t batch, int32_t total_q, float scale,
+                     void* out, void* workspace, size_t workspace_bytes, int32_t kv_split_tokens,
+                     int32_t* dev_status, void* cuda_stream);
+/* What the calling thread's last pa_prefill / pa_prefill_split launched: row tiles per CTA (0 =
+ * the warp-level kernel), split length in tokens (0 = unsplit) and partial rows per query row.
+ * A measurement and test aid; no counterpart in the paper. */
+int pa_prefill_last_launch(int32_t* tiles_per_cta, int32_t* kv_split_tokens, int32_t* kv_splits);
+
+/*
  * KV append (Section 2.2 "KV-Cache": with every decoding step the KV vectors of the newly
  * generated token are appended to the cache).  For every b < batch with slot_mapping[b] >= 0
  * the rows k_new[b,:,:] and v_new[b,:,:] are written to slot (slot_mapping[b] % block_size)

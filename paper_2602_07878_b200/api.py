@@ -32,7 +32,8 @@ EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_hos
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
            "pa_decode_static", "kv_append", "pa_partial_floats", "pa_decode_partial",
            "pa_merge_partials",
-           "pa_prefill_workspace_bytes", "pa_prefill", "pa_selftest_wait_expiry", "pa_probe_read"]
+           "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_split",
+           "pa_prefill_split_workspace_bytes", "pa_prefill_last_launch", "pa_selftest_wait_expiry", "pa_probe_read"]
 
 
 class PaShape(ctypes.Structure):
@@ -88,6 +89,14 @@ def lib() -> ctypes.CDLL:
         L.pa_prefill.argtypes = [pshape, vp, vp, vp, vp, i32, vp, vp, i32, i32, ctypes.c_float, vp,
                                  vp, sz, vp, vp]
         L.pa_prefill.restype = ctypes.c_int
+        L.pa_prefill_split.argtypes = [pshape, vp, vp, vp, vp, i32, vp, vp, i32, i32,
+                                       ctypes.c_float, vp, vp, sz, i32, vp, vp]
+        L.pa_prefill_split.restype = ctypes.c_int
+        L.pa_prefill_split_workspace_bytes.argtypes = [pshape, i32, i32, i32, psz]
+        L.pa_prefill_split_workspace_bytes.restype = ctypes.c_int
+        pi32 = ctypes.POINTER(ctypes.c_int32)
+        L.pa_prefill_last_launch.argtypes = [pi32, pi32, pi32]
+        L.pa_prefill_last_launch.restype = ctypes.c_int
         L.pa_selftest_wait_expiry.argtypes = [i32, vp, vp]
         L.pa_selftest_wait_expiry.restype = ctypes.c_int
         L.pa_probe_read.argtypes = [vp, sz, i32, ctypes.c_uint32, vp, vp, vp]
@@ -338,21 +347,58 @@ def pa_prefill_workspace_bytes(max_batch: int) -> int:
     return int(out.value)
 
 
-def pa_prefill(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, out, workspace, *,
-               dev_status=None, stream=None):
-    """Forward to pa_prefill.  q/out [total_q,H,D] bf16 (packed tokens); ctx_lens int32 [B];
-    cu_q_lens int32 [B+1]; caches and block_tables as for pa_decode."""
+def pa_prefill_split_workspace_bytes(shape: PaShape, max_batch: int, max_total_q: int,
+                                     max_splits: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().pa_prefill_split_workspace_bytes(ctypes.byref(shape), max_batch, max_total_q,
+                                                  max_splits, ctypes.byref(out)),
+           "pa_prefill_split_workspace_bytes")
+    return int(out.value)
+
+
+def pa_prefill_last_launch():
+    """Forward to pa_prefill_last_launch: (tiles per CTA, split tokens, partial rows per row)."""
+    a, b, c = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(lib().pa_prefill_last_launch(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+           "pa_prefill_last_launch")
+    return a.value, b.value, c.value
+
+
+def _prefill_args(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, out):
     shape = shape_of(k_cache, q.shape[1])
     assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
     assert block_tables.dtype == torch.int32 and ctx_lens.dtype == torch.int32
     assert cu_q_lens.dtype == torch.int32 and cu_q_lens.numel() == ctx_lens.numel() + 1
     assert q.is_contiguous() and out.is_contiguous() and block_tables.is_contiguous()
+    return shape
+
+
+def pa_prefill(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, out, workspace, *,
+               dev_status=None, stream=None):
+    """Forward to pa_prefill.  q/out [total_q,H,D] bf16 (packed tokens); ctx_lens int32 [B];
+    cu_q_lens int32 [B+1]; caches and block_tables as for pa_decode."""
+    shape = _prefill_args(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, out)
     rc = lib().pa_prefill(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
                           _ptr(block_tables), block_tables.shape[1], _ptr(ctx_lens),
                           _ptr(cu_q_lens), ctx_lens.numel(), q.shape[0], float(scale), _ptr(out),
                           _ptr(workspace), workspace.numel() * workspace.element_size(),
                           _ptr(dev_status), _stream(stream))
     _check(rc, "pa_prefill")
+    return out
+
+
+def pa_prefill_split(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, out,
+                     workspace, *, kv_split_tokens=0, dev_status=None, stream=None):
+    """Forward to pa_prefill_split: pa_prefill with the KV range split over CTAs
+    (kv_split_tokens: 0 = chosen by the library, > 0 = forced, < 0 = never)."""
+    shape = _prefill_args(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, out)
+    rc = lib().pa_prefill_split(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                _ptr(block_tables), block_tables.shape[1], _ptr(ctx_lens),
+                                _ptr(cu_q_lens), ctx_lens.numel(), q.shape[0], float(scale),
+                                _ptr(out), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(),
+                                int(kv_split_tokens), _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_prefill_split")
     return out
 
 

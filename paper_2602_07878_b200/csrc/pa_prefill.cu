@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdlib>
 #include <mutex>
 #include <string>
@@ -23,12 +24,20 @@ struct PrefillPlanParams {
     const int32_t* ctx_lens;
     const int32_t* cu_q_lens;
     int batch, max_blocks, total_q, tpg;  // tpg = query tokens per 16-row group
+    int split_steps;  // KV range of one unit in 64-token steps (0 = the whole context)
     int* hdr;
     int* gstart;  // [batch + 1] first group of each sequence
     int* status;
 };
 
-// one CTA: validate lengths, count 16-row groups per sequence, exclusive scan
+// number of KV splits of a sequence with L cached tokens when a unit covers T 64-token steps
+__host__ __device__ __forceinline__ int kv_splits(int L, int T) {
+    if (T <= 0 || L <= 0) return 1;
+    const int steps = (L - 1) / 64 + 1;
+    return (steps + T - 1) / T;
+}
+
+// one CTA: validate lengths, count units (row groups x KV splits) per sequence, exclusive scan
 __global__ void __launch_bounds__(1024, 1) pa_prefill_plan_kernel(const PrefillPlanParams p) {
     __shared__ int warp_sums[32];
     __shared__ int s_carry, s_bad;
@@ -44,7 +53,7 @@ __global__ void __launch_bounds__(1024, 1) pa_prefill_plan_kernel(const PrefillP
             const bool ok = q0 >= 0 && ql >= 0 && q1 <= p.total_q && L >= ql &&
                             L <= p.max_blocks * BS && (b > 0 || q0 == 0);
             if (!ok) s_bad = 1;
-            n = ok ? (ql + p.tpg - 1) / p.tpg : 0;
+            n = ok ? (ql + p.tpg - 1) / p.tpg * kv_splits(L, p.split_steps) : 0;
         }
         int incl = n;
         for (int o = 1; o < 32; o <<= 1) {
@@ -298,6 +307,14 @@ enum { T_SFULL = 0, T_PFULL = 2, T_PVDONE = 4 };
 struct PrefillTcParams {
     PrefillParams base;
     int tokens_per_tile;  // 128 / G
+    // KV split: a unit covers `split_steps` 64-token steps of its tile's visible context (0 =
+    // all of it).  A sequence with more than one split leaves, per (query row, split), an
+    // un-normalised fp32 output row in part_o[(row * split_cap + s) * D] and its reference
+    // exponent and weight sum in part_ml[(row * split_cap + s) * 2]; row = query token * H +
+    // head.  A negative sum marks a split that met a bad block id.
+    int split_steps, split_cap;
+    float* part_ml;
+    float* part_o;
 };
 
 template <int NT>
@@ -335,10 +352,15 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     }
     const int b = lo;
     const int q0 = p.cu_q_lens[b], ql = p.cu_q_lens[b + 1] - q0, L = p.ctx_lens[b];
-    const int tok0 = (gi - p.gstart[b]) * (NT * tpt);   // first query token of the CTA
+    const int n_split = kv_splits(L, tp.split_steps);   // units per row group of this sequence
+    const int r = gi - p.gstart[b];
+    const int split = r % n_split;
+    const int tok0 = (r / n_split) * (NT * tpt);        // first query token of the CTA
     const int ntok_cta = min(NT * tpt, ql - tok0);
     const int pos_max = L - ql + tok0 + ntok_cta - 1;
-    const int n_steps = pos_max / STEP + 1;
+    const int j0 = split * tp.split_steps;              // first 64-token step of this unit
+    const int n_steps = min(pos_max / STEP + 1 - j0, n_split > 1 ? tp.split_steps : 0x7fffffff);
+    if (n_steps <= 0) return;                           // the tile sees nothing of this split
     const int nblk_seq = (L + BS - 1) / BS;
 
     if (tid == 0) {
@@ -384,13 +406,15 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             }
         }
         const int32_t* table = p.block_tables + (size_t)b * p.max_blocks;
-        int ids = lane < nblk_seq ? __ldg(&table[lane]) : p.NB;
-        int ids_next = 32 + lane < nblk_seq ? __ldg(&table[32 + lane]) : p.NB;
+        // block ids are fetched 32 at a time, one window ahead; the unit starts at block 4 * j0
+        const int win0 = (j0 * 4) & ~31;
+        int ids = win0 + lane < nblk_seq ? __ldg(&table[win0 + lane]) : p.NB;
+        int ids_next = win0 + 32 + lane < nblk_seq ? __ldg(&table[win0 + 32 + lane]) : p.NB;
         for (int j = 0; j < n_steps; ++j) {
             const int stage = j % ST;
             if (j >= ST && !wait(B_KVEMPTY + stage, ((j / ST) - 1) & 1)) break;
-            const int blk0 = j * 4;
-            if (blk0 > 0 && (blk0 & 31) == 0) {
+            const int blk0 = (j0 + j) * 4;
+            if (blk0 > win0 && (blk0 & 31) == 0) {
                 ids = ids_next;
                 ids_next = blk0 + 32 + lane < nblk_seq ? __ldg(&table[blk0 + 32 + lane]) : p.NB;
             }
@@ -488,7 +512,7 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             tmem_ld32(tcol + lane_base + (j & 1) * STEP + 32, sr[1]);
             tmem_wait_ld();
 
-            const int t0 = j * STEP;
+            const int t0 = (j0 + j) * STEP;
             uint32_t pk[STEP / 2];
             float corr = 1.f, lsum = 0.f;
             if (sl2 > 0.f) {
@@ -592,9 +616,29 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(tb + T_PFULL + (j & 1)));
         }
-        // ---- epilogue: O / l -> bf16 rows ----
+        // ---- epilogue: O / l -> bf16 rows, or the unit's partial record when the KV is split ----
         if (ok) ok = wait(tb + T_PVDONE + ((n_steps - 1) & 1), ((n_steps - 1) >> 1) & 1);
-        if (ok) {
+        if (ok && n_split > 1) {
+            tc_fence_after_sync();
+            const size_t rec =
+                ((size_t)(q0 + qtok) * H + (size_t)kvh * G + hd) * tp.split_cap + split;
+            if (row_ok)
+                *reinterpret_cast<float2*>(tp.part_ml + rec * 2) =
+                    make_float2(m_ref, misc[2] != 0 ? -1.f : l);
+            float* dst = tp.part_o + rec * D;
+#pragma unroll 1
+            for (int c = 0; c < D; c += 32) {
+                uint32_t o[32];
+                tmem_ld32(tcol + lane_base + 2 * STEP + c, o);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<uint4*>(dst + c + i) =
+                            make_uint4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                }
+            }
+        } else if (ok) {
             tc_fence_after_sync();
             const bool bad = misc[2] != 0;
             const float inv = bad ? 0.f : 1.f / l;
@@ -626,6 +670,76 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
+}
+
+struct PrefillMergeParams {
+    const int32_t* ctx_lens;
+    const int32_t* cu_q_lens;
+    const float* part_ml;
+    const float* part_o;
+    __nv_bfloat16* out;
+    int batch, max_blocks, total_q, H, tpg, split_steps, split_cap;
+};
+
+// Merge of the KV splits of pa_prefill_tc_kernel: one warp per (query token, head) row.
+//   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,   M = max_s m_s
+// over the splits the row's tile has visited.  Rows of sequences with a single split were
+// written by the attention kernel itself and are skipped, as are rows of refused sequences.
+__global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMergeParams p) {
+    constexpr int D = 128;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= (long long)p.total_q * p.H) return;
+    const int qi = (int)(row / p.H);
+    int lo = 0, hi = p.batch;  // last b with cu_q_lens[b] <= qi
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(&p.cu_q_lens[mid]) <= qi) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int q0 = __ldg(&p.cu_q_lens[b]), q1 = __ldg(&p.cu_q_lens[b + 1]), L = __ldg(&p.ctx_lens[b]);
+    const int ql = q1 - q0;
+    const bool ok = q0 >= 0 && ql >= 0 && q1 <= p.total_q && L >= ql &&
+                    L <= p.max_blocks * BS && (b > 0 || q0 == 0) && qi >= q0 && qi < q1;
+    if (!ok) return;
+    const int n_split = kv_splits(L, p.split_steps);
+    if (n_split <= 1) return;
+    // splits visited by the row's tile group: those that start at or before its last position
+    const int tok0 = (qi - q0) / p.tpg * p.tpg;
+    const int pos_max = L - ql + min(tok0 + p.tpg, ql) - 1;
+    const int n_vis = min(n_split, (pos_max / 64 + 1 + p.split_steps - 1) / p.split_steps);
+    const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + (size_t)row * p.split_cap;
+    float M = -INFINITY;
+    bool bad = false;
+    for (int s = lane; s < n_vis; s += 32) {
+        const float2 v = ml[s];
+        M = fmaxf(M, v.x);
+        bad |= v.y < 0.f;
+    }
+    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    bad = __any_sync(0xffffffffu, bad);
+    const float4* po = reinterpret_cast<const float4*>(p.part_o) + (size_t)row * p.split_cap * (D / 4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lsum = 0.f;
+#pragma unroll 4
+    for (int s = 0; s < n_vis; ++s) {
+        const float2 v = ml[s];
+        const float4 o = po[(size_t)s * (D / 4) + lane];
+        const float w = v.x == -INFINITY ? 0.f : ex2(v.x - M);
+        acc.x = fmaf(w, o.x, acc.x);
+        acc.y = fmaf(w, o.y, acc.y);
+        acc.z = fmaf(w, o.z, acc.z);
+        acc.w = fmaf(w, o.w, acc.w);
+        lsum = fmaf(w, v.y, lsum);
+    }
+    const float inv = (bad || !(lsum > 0.f)) ? 0.f : 1.f / lsum;
+    uint2 w;
+    w.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    w.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    if (bad) w = make_uint2(0u, 0u);
+    reinterpret_cast<uint2*>(p.out + (size_t)row * D)[lane] = w;
 }
 
 // tensor map over the packed queries viewed as [total_q][Hkv][G][D]: box 64 x G x 1 x (128/G)
@@ -696,19 +810,87 @@ static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const
 
 using namespace pk;
 
+static size_t prefill_base_bytes(int64_t batch) {
+    const size_t b = PF_WORDS * sizeof(int) + ((size_t)batch + 1) * sizeof(int) + 256;
+    return (b + 255) & ~(size_t)255;
+}
+
 extern "C" int pa_prefill_workspace_bytes(int32_t max_batch, size_t* bytes) {
     if (!bytes) return PA_ERR_NULL;
     if (max_batch < 0) return PA_ERR_ARG;
-    *bytes = PF_WORDS * sizeof(int) + ((size_t)max_batch + 1) * sizeof(int) + 256;
+    *bytes = prefill_base_bytes(max_batch);
     return PA_OK;
 }
 
-extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache,
-                          const void* v_cache, const int32_t* block_tables,
-                          int32_t max_blocks_per_seq, const int32_t* ctx_lens,
-                          const int32_t* cu_q_lens, int32_t batch, int32_t total_q, float scale,
-                          void* out, void* workspace, size_t workspace_bytes, int32_t* dev_status,
-                          void* cuda_stream) {
+extern "C" int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t max_batch,
+                                                int32_t max_total_q, int32_t max_splits,
+                                                size_t* bytes) {
+    if (!bytes || !shape) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (max_batch < 0 || max_total_q < 0 || max_splits < 1) return PA_ERR_ARG;
+    *bytes = prefill_base_bytes(max_batch) + (size_t)max_total_q * shape->num_q_heads *
+                                                 max_splits * (shape->head_dim + 2) * sizeof(float);
+    return PA_OK;
+}
+
+namespace pk {
+// Launch shape of the tensor-core path: row tiles per CTA and the KV split length in 64-token
+// steps (0 = no split).  Only bounds are known on the host (the chunk's token count, the
+// longest context the block table can describe), so this is a cost model, not a plan: rounds
+// of CTAs over the SMs times the steps of one unit, a fixed cost per unit, and the traffic of
+// the partial records when the KV range is split.
+struct TcShape {
+    int tiles_per_cta, split_steps, split_cap;
+};
+static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H, int D,
+                               int64_t steps_bound, int sm_count, int64_t cap_fit,
+                               int forced_tiles, int forced_split_steps) {
+    const int tpt = 128 / G;
+    TcShape best = {1, 0, 1};
+    double best_t = 1e30;
+    for (int nt = 1; nt <= 2; ++nt) {
+        if (forced_tiles && nt != forced_tiles) continue;
+        const int64_t tpg = (int64_t)nt * tpt;
+        const int64_t groups =
+            (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
+        // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
+        // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
+        const double step_us = nt == 1 ? 0.83 : 1.28;
+        const int64_t s_hi = forced_split_steps ? 1 : std::min<int64_t>({cap_fit, 64, steps_bound / 8});
+        for (int64_t s_try = 1; s_try <= std::max<int64_t>(1, s_hi); ++s_try) {
+            int64_t T = forced_split_steps ? forced_split_steps : (steps_bound + s_try - 1) / s_try;
+            const int64_t S = (steps_bound + T - 1) / T;
+            if (S > cap_fit && S > 1) continue;
+            const int64_t rounds = (groups * S + sm_count - 1) / sm_count;
+            double t = rounds * (T * step_us + 4.0);
+            if (S > 1) t += 6.0 + (double)total_q * H * S * (D + 2) * 4 * 2 / 2.5e6;
+            if (t < best_t) {
+                best_t = t;
+                best = {nt, S > 1 ? (int)T : 0, (int)std::max<int64_t>(S, 1)};
+            }
+        }
+    }
+    return best;
+}
+static thread_local TcShape g_last_shape = {0, 0, 1};
+}  // namespace pk
+
+extern "C" int pa_prefill_last_launch(int32_t* tiles_per_cta, int32_t* kv_split_tokens,
+                                      int32_t* kv_splits) {
+    if (!tiles_per_cta || !kv_split_tokens || !kv_splits) return PA_ERR_NULL;
+    *tiles_per_cta = g_last_shape.tiles_per_cta;
+    *kv_split_tokens = g_last_shape.split_steps * 64;
+    *kv_splits = g_last_shape.split_cap;
+    return PA_OK;
+}
+
+extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void* k_cache,
+                                const void* v_cache, const int32_t* block_tables,
+                                int32_t max_blocks_per_seq, const int32_t* ctx_lens,
+                                const int32_t* cu_q_lens, int32_t batch, int32_t total_q,
+                                float scale, void* out, void* workspace, size_t workspace_bytes,
+                                int32_t kv_split_tokens, int32_t* dev_status, void* cuda_stream) {
     if (!shape) return PA_ERR_NULL;
     int rc = validate_shape(shape);
     if (rc) return rc;
@@ -721,9 +903,8 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
         return PA_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return PA_ERR_ALIGN;
     if ((int64_t)max_blocks_per_seq * BS > INT32_MAX) return PA_ERR_ARG;
-    size_t need = 0;
-    pa_prefill_workspace_bytes(batch, &need);
-    if (workspace_bytes < need) return PA_ERR_WORKSPACE;
+    const size_t base_bytes = prefill_base_bytes(batch);
+    if (workspace_bytes < base_bytes) return PA_ERR_WORKSPACE;
     DeviceInfo dev;
     rc = get_device_info(&dev);
     if (rc) return rc;
@@ -735,6 +916,7 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int* hdr = static_cast<int*>(workspace);
     const int G = shape->num_q_heads / shape->num_kv_heads;
+    const int H = shape->num_q_heads, D = shape->head_dim;
 
     PrefillPlanParams plan;
     plan.ctx_lens = ctx_lens;
@@ -747,20 +929,33 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
         const char* e = std::getenv("PAGEDKV_PREFILL");
         return e && std::string(e) == "mma";
     }();
-    const bool use_tc = !force_mma && shape->head_dim == 128 && (128 % G) == 0;
-    // two row tiles per CTA (two softmax warpgroups sharing the K/V stages) once there are
-    // enough tiles to still give every SM a CTA; otherwise one tile per CTA
+    const bool use_tc = !force_mma && D == 128 && (128 % G) == 0;
     static const int forced_tiles = [] {
         const char* e = std::getenv("PAGEDKV_PREFILL_TILES");
-        return e ? std::atoi(e) : 0;
+        const int v = e ? std::atoi(e) : 0;
+        return v == 1 || v == 2 ? v : 0;
     }();
-    int tiles_per_cta = 1;
+    TcShape ts = {1, 0, 1};
     if (use_tc) {
-        const int64_t tiles = ((int64_t)total_q / (128 / G) + batch) * shape->num_kv_heads;
-        tiles_per_cta = tiles >= 2LL * dev.sm_count ? 2 : 1;
-        if (forced_tiles == 1 || forced_tiles == 2) tiles_per_cta = forced_tiles;
+        const int64_t steps_bound = std::max<int64_t>(1, ((int64_t)max_blocks_per_seq * BS + 63) / 64);
+        const size_t per_split = (size_t)total_q * H * (D + 2) * sizeof(float);
+        const int64_t cap_fit = (int64_t)((workspace_bytes - base_bytes) / per_split);
+        int forced_steps = 0;
+        if (kv_split_tokens > 0) {
+            forced_steps = (kv_split_tokens + 63) / 64;
+            if (forced_steps >= steps_bound) kv_split_tokens = -1;  // one split covers everything
+            else if ((steps_bound + forced_steps - 1) / forced_steps > cap_fit) return PA_ERR_WORKSPACE;
+        }
+        if (kv_split_tokens < 0)
+            ts = choose_tc_shape(total_q, batch, shape->num_kv_heads, G, H, D, steps_bound,
+                                 dev.sm_count, 1, forced_tiles, 0);
+        else
+            ts = choose_tc_shape(total_q, batch, shape->num_kv_heads, G, H, D, steps_bound,
+                                 dev.sm_count, cap_fit, forced_tiles, forced_steps);
     }
-    plan.tpg = use_tc ? tiles_per_cta * (128 / G) : 16 / G;
+    g_last_shape = use_tc ? ts : TcShape{0, 0, 1};
+    plan.tpg = use_tc ? ts.tiles_per_cta * (128 / G) : 16 / G;
+    plan.split_steps = ts.split_steps;
     plan.hdr = hdr;
     plan.gstart = hdr + PF_WORDS;
     plan.status = dev_status ? dev_status : hdr + PF_STATUS;
@@ -780,7 +975,7 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
     pp.status = plan.status;
     pp.batch = batch;
     pp.max_blocks = max_blocks_per_seq;
-    pp.H = shape->num_q_heads;
+    pp.H = H;
     pp.Hkv = shape->num_kv_heads;
     pp.G = G;
     pp.NB = shape->num_blocks;
@@ -788,16 +983,57 @@ extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_ca
     pp.scale_log2 = scale * 1.4426950408889634f;
     if (use_tc) {
         CUtensorMap qm;
-        rc = make_q_map(&qm, q, total_q, pp.Hkv, G, shape->head_dim);
+        rc = make_q_map(&qm, q, total_q, pp.Hkv, G, D);
         if (rc) return rc;
         PrefillTcParams tp;
         tp.base = pp;
         tp.tokens_per_tile = 128 / G;
-        const int max_ctas = (total_q / plan.tpg + batch) * pp.Hkv;
-        return tiles_per_cta == 2 ? launch_prefill_tc<2>(qm, km, vm, tp, max_ctas, dev, st)
-                                  : launch_prefill_tc<1>(qm, km, vm, tp, max_ctas, dev, st);
+        tp.split_steps = ts.split_steps;
+        tp.split_cap = ts.split_cap;
+        tp.part_ml = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + base_bytes);
+        tp.part_o = tp.part_ml + (size_t)total_q * H * ts.split_cap * 2;
+        const int64_t max_ctas = ((int64_t)total_q / plan.tpg + batch) * pp.Hkv * ts.split_cap;
+        if (max_ctas > INT32_MAX) return PA_ERR_ARG;
+        rc = ts.tiles_per_cta == 2 ? launch_prefill_tc<2>(qm, km, vm, tp, (int)max_ctas, dev, st)
+                                   : launch_prefill_tc<1>(qm, km, vm, tp, (int)max_ctas, dev, st);
+        if (rc || ts.split_steps == 0) return rc;
+        PrefillMergeParams mp;
+        mp.ctx_lens = ctx_lens;
+        mp.cu_q_lens = cu_q_lens;
+        mp.part_ml = tp.part_ml;
+        mp.part_o = tp.part_o;
+        mp.out = pp.out;
+        mp.batch = batch;
+        mp.max_blocks = max_blocks_per_seq;
+        mp.total_q = total_q;
+        mp.H = H;
+        mp.tpg = plan.tpg;
+        mp.split_steps = ts.split_steps;
+        mp.split_cap = ts.split_cap;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(((int64_t)total_q * H + 7) / 8));
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        count_launch();
+        return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel, mp));
     }
-    return shape->head_dim == 256   ? launch_prefill<256>(km, vm, pp, dev, st)
-           : shape->head_dim == 128 ? launch_prefill<128>(km, vm, pp, dev, st)
-                                    : launch_prefill<64>(km, vm, pp, dev, st);
+    return D == 256   ? launch_prefill<256>(km, vm, pp, dev, st)
+           : D == 128 ? launch_prefill<128>(km, vm, pp, dev, st)
+                      : launch_prefill<64>(km, vm, pp, dev, st);
+}
+
+extern "C" int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache,
+                          const void* v_cache, const int32_t* block_tables,
+                          int32_t max_blocks_per_seq, const int32_t* ctx_lens,
+                          const int32_t* cu_q_lens, int32_t batch, int32_t total_q, float scale,
+                          void* out, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                          void* cuda_stream) {
+    return pa_prefill_split(shape, q, k_cache, v_cache, block_tables, max_blocks_per_seq, ctx_lens,
+                            cu_q_lens, batch, total_q, scale, out, workspace, workspace_bytes, 0,
+                            dev_status, cuda_stream);
 }

@@ -12,22 +12,29 @@ pytestmark = pytest.mark.gpu
 
 
 class GpuPrefill:
-    def __init__(self, spec, q_bits, k_bits, v_bits):
+    def __init__(self, spec, q_bits, k_bits, v_bits, max_splits=0):
         self.spec = spec
         self.q = bits_to_torch(q_bits)
         self.k, self.v = bits_to_torch(k_bits), bits_to_torch(v_bits)
         self.tables = torch.from_numpy(spec.block_tables).cuda()
-        self.ws = torch.empty(api.pa_prefill_workspace_bytes(spec.batch), dtype=torch.uint8,
-                              device="cuda")
+        nbytes = api.pa_prefill_workspace_bytes(spec.batch)
+        if max_splits:
+            nbytes = api.pa_prefill_split_workspace_bytes(
+                api.shape_of(self.k, q_bits.shape[1]), spec.batch, q_bits.shape[0], max_splits)
+        # NaN-filled: a partial record that is read without having been written shows up
+        self.ws = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
 
-    def run(self, ctx, cu, q=None, tables=None):
+    def run(self, ctx, cu, q=None, tables=None, split=None):
         q = self.q if q is None else q
         out = torch.full_like(q, float("nan"))
-        api.pa_prefill(q, self.k, self.v, self.tables if tables is None else tables,
-                       torch.from_numpy(np.asarray(ctx, np.int32)).cuda(),
-                       torch.from_numpy(np.asarray(cu, np.int32)).cuda(), self.spec.scale, out,
-                       self.ws, dev_status=self.status)
+        args = (q, self.k, self.v, self.tables if tables is None else tables,
+                torch.from_numpy(np.asarray(ctx, np.int32)).cuda(),
+                torch.from_numpy(np.asarray(cu, np.int32)).cuda(), self.spec.scale, out, self.ws)
+        if split is None:
+            api.pa_prefill(*args, dev_status=self.status)
+        else:
+            api.pa_prefill_split(*args, kv_split_tokens=split, dev_status=self.status)
         torch.cuda.synchronize()
         return out
 
@@ -124,11 +131,91 @@ def test_large_scores_and_growing_maxima():
 
 
 def test_large_chunk_takes_the_two_tile_kernel():
-    # (1300 / 32 + 2) * 8 KV heads = 336 tiles >= 2 x 148 SMs: two row tiles per CTA, two
-    # softmax warpgroups sharing the K/V stages; the second sequence ends in a half-used pair
-    spec, q, k, v, cu = make_case([1500, 777], [900, 400], 32, 8, 128, seed=60)
+    # (2300 / 64 + 2) * 8 KV heads = 296 CTAs of two row tiles fill two rounds of 148 SMs: two
+    # softmax warpgroups share the K/V stages; the second sequence ends in a half-used pair
+    spec, q, k, v, cu = make_case([2100, 1201], [1500, 800], 32, 8, 128, seed=60)
     g = GpuPrefill(spec, q, k, v)
     out = torch_to_f64(g.run(spec.seq_lens, cu))
+    assert api.pa_prefill_last_launch() == (2, 0, 1)
     ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
     assert int(g.status.item()) == 0
     assert_parity(out, ref, "two tiles per CTA")
+
+
+# ---- KV range split over CTAs (pa_prefill_split) --------------------------------------------
+
+@pytest.mark.parametrize("H,Hkv", [(4, 4), (32, 8), (16, 1)])
+@pytest.mark.parametrize("split", [64, 192, 1024])
+def test_forced_kv_split_matches_oracle(H, Hkv, split):
+    # contexts that end inside a block and inside a split, tiles whose last rows see fewer
+    # splits than the sequence has, a sequence that fits one split (written directly), an
+    # empty chunk
+    ctx = [4999, 130, 1031, 64, 300]
+    qlens = [517, 130, 7, 1, 0]
+    spec, q, k, v, cu = make_case(ctx, qlens, H, Hkv, 128, seed=70 + H)
+    max_splits = -(-spec.block_tables.shape[1] * 16 // split)
+    g = GpuPrefill(spec, q, k, v, max_splits=max_splits)
+    out = g.run(spec.seq_lens, cu, split=split)
+    tiles, tok, cap = api.pa_prefill_last_launch()
+    assert tiles in (1, 2) and tok == split and cap == max_splits
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(torch_to_f64(out), ref, f"H{H}/{Hkv} split {split}")
+    again = g.run(spec.seq_lens, cu, split=split)
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16))
+
+
+def test_kv_split_with_two_tiles_per_cta():
+    # enough query tokens for two row tiles per CTA; queries in the middle of the context, so
+    # the first tiles end before the last splits begin
+    spec, q, k, v, cu = make_case([2600, 1111], [1500, 900], 32, 8, 128, seed=80)
+    split = 512
+    max_splits = -(-spec.block_tables.shape[1] * 16 // split)
+    g = GpuPrefill(spec, q, k, v, max_splits=max_splits)
+    out = torch_to_f64(g.run(spec.seq_lens, cu, split=split))
+    assert api.pa_prefill_last_launch() == (2, split, max_splits)
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, "split, two tiles per CTA")
+
+
+def test_library_chosen_split_on_a_recompute_chunk():
+    # one long victim, the last 256 tokens of a 6000-token context: 16 tiles for 148 SMs, so
+    # the library splits the KV range by itself once the workspace allows it
+    spec, q, k, v, cu = make_case([6000], [256], 8, 2, 128, seed=81)
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    g = GpuPrefill(spec, q, k, v, max_splits=16)
+    out = torch_to_f64(g.run(spec.seq_lens, cu, split=0))
+    tiles, tok, cap = api.pa_prefill_last_launch()
+    assert tok > 0 and 1 < cap <= 16, (tiles, tok, cap)
+    assert_parity(out, ref, "library-chosen split")
+    # the same call with a workspace that holds no partial rows runs unsplit
+    g1 = GpuPrefill(spec, q, k, v)
+    out1 = torch_to_f64(g1.run(spec.seq_lens, cu))
+    assert api.pa_prefill_last_launch()[1:] == (0, 1)
+    assert_parity(out1, ref, "unsplit")
+    assert int(g.status.item()) == 0 and int(g1.status.item()) == 0
+    # never split on request
+    g.run(spec.seq_lens, cu, split=-1)
+    assert api.pa_prefill_last_launch()[1:] == (0, 1)
+
+
+def test_kv_split_errors():
+    spec, q, k, v, cu = make_case([2000, 640], [64, 640], 8, 2, 128, seed=82)
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    g = GpuPrefill(spec, q, k, v, max_splits=2)
+    with pytest.raises(api.PagedKVError) as e:       # 2000 tokens in 256-token splits: 8 rows
+        g.run(spec.seq_lens, cu, split=256)
+    assert e.value.code == api.ERR["WORKSPACE"]
+    g = GpuPrefill(spec, q, k, v, max_splits=8)
+    t = spec.block_tables.copy()
+    t[0, 40] = spec.num_blocks + 3                   # tokens 640..655 of sequence 0: split 2
+    out = torch_to_f64(g.run(spec.seq_lens, cu, tables=torch.from_numpy(t).cuda(), split=256))
+    assert int(g.status.item()) == api.PA_STATUS_BAD_BLOCK_ID
+    assert (out[:64] == 0).all()                     # every query of sequence 0 sees block 40
+    assert_parity(out[64:], ref[64:])
+    g.status.zero_()
+    out = torch_to_f64(g.run([2000, 600], cu, split=256))   # ctx < q_len for sequence 1
+    assert int(g.status.item()) == api.PA_STATUS_BAD_SEQ_LEN
+    assert np.isnan(out[64:]).all()
+    assert_parity(out[:64], ref[:64])
