@@ -437,56 +437,64 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             }
         }
     } else if (warp == C::MMA_WARP) {
-        // ===================== MMA issuer (one thread) =====================
+        // ===================== MMA issuer =====================
+        // The whole warp walks the loop and one elected lane issues: descriptor arithmetic
+        // that is uniform across the warp stays off the issuing lane's critical path (issued
+        // from a single-lane branch an MMA costs 50-65 cycles of issue, this way 30-40).
         // Per step j: Q K^T of step j for every tile, then P V of step j-1 for every tile, so
         // that the tensor pipe always has the other tile's work while one tile is in softmax.
         // S(j % 2) is free for Q K^T of step j once P V of step j-2, which read its weights
         // from there, has been issued: MMAs of one thread execute in issue order.
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = tc_idesc_bf16(ROWS, STEP, false);
-            constexpr uint32_t idesc_pv = tc_idesc_bf16(ROWS, D, true);
-            bool ok = wait(B_QFULL, 0);
-            for (int j = 0; ok && j <= n_steps; ++j) {
-                if (j < n_steps) {  // S[tile][j % 2] = Q_tile K_j^T
-                    const int stage = j % ST;
-                    ok = wait(B_KVFULL + stage, (j / ST) & 1);
-                    const uint32_t kb = sbase + OFF_KV + stage * STAGE_BYTES;
-                    for (int t = 0; ok && t < NT; ++t) {
-                        const int tb = C::B_TILE + 8 * t;
-                        const uint32_t qb = sbase + OFF_Q + t * Q_BYTES;
+        constexpr uint32_t idesc_qk = tc_idesc_bf16(ROWS, STEP, false);
+        constexpr uint32_t idesc_pv = tc_idesc_bf16(ROWS, D, true);
+        auto wait_all = [&](int b_idx, uint32_t parity) -> bool {
+            return __all_sync(0xffffffffu, wait(b_idx, parity));
+        };
+        bool ok = wait_all(B_QFULL, 0);
+        for (int j = 0; ok && j <= n_steps; ++j) {
+            if (j < n_steps) {  // S[tile][j % 2] = Q_tile K_j^T
+                const int stage = j % ST;
+                ok = wait_all(B_KVFULL + stage, (j / ST) & 1);
+                if (!ok) break;
+                const uint32_t kb = sbase + OFF_KV + stage * STAGE_BYTES;
 #pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks) {
-                            const uint64_t a =
-                                tc_smem_desc(qb + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32, 16, 1024);
-                            const uint64_t bd =
-                                tc_smem_desc(kb + (ks >> 2) * KV_HALF + (ks & 3) * 32, 16, 1024);
+                for (int t = 0; t < NT; ++t) {
+                    const int tb = C::B_TILE + 8 * t;
+                    const uint32_t qb = sbase + OFF_Q + t * Q_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint64_t a =
+                            tc_smem_desc(qb + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32, 16, 1024);
+                        const uint64_t bd =
+                            tc_smem_desc(kb + (ks >> 2) * KV_HALF + (ks & 3) * 32, 16, 1024);
+                        if (elect_one())
                             tc_mma_bf16(tmem + t * 256 + (j & 1) * STEP, a, bd, idesc_qk, ks > 0);
-                        }
-                        tc_commit(bar(tb + T_SFULL + (j & 1)));
                     }
-                    if (!ok) break;
+                    if (elect_one()) tc_commit(bar(tb + T_SFULL + (j & 1)));
                 }
-                if (j >= 1) {  // O[tile] += P_{j-1} V_{j-1}
-                    const int i = j - 1, stage = i % ST;
-                    const uint32_t vb = sbase + OFF_KV + stage * STAGE_BYTES + 2 * KV_HALF;
-                    for (int t = 0; ok && t < NT; ++t) {
-                        const int tb = C::B_TILE + 8 * t;
-                        ok = wait(tb + T_PFULL + (i & 1), (i >> 1) & 1);
-                        if (!ok) break;
-                        tc_fence_after_sync();
-                        const uint32_t pt = tmem + t * 256 + (i & 1) * STEP;
+            }
+            if (j >= 1) {  // O[tile] += P_{j-1} V_{j-1}
+                const int i = j - 1, stage = i % ST;
+                const uint32_t vb = sbase + OFF_KV + stage * STAGE_BYTES + 2 * KV_HALF;
 #pragma unroll
-                        for (int kk = 0; kk < STEP / 16; ++kk) {
-                            // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
-                            const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
+                for (int t = 0; t < NT; ++t) {
+                    const int tb = C::B_TILE + 8 * t;
+                    ok = ok && wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t pt = tmem + t * 256 + (i & 1) * STEP;
+#pragma unroll
+                    for (int kk = 0; kk < STEP / 16; ++kk) {
+                        // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
+                        const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
+                        if (elect_one())
                             tc_mma_bf16_ta(tmem + t * 256 + 2 * STEP, pt + kk * 8, bd, idesc_pv,
                                            (i > 0 || kk > 0) ? 1u : 0u);
-                        }
-                        tc_commit(bar(tb + T_PVDONE + (i & 1)));
                     }
-                    if (!ok) break;
-                    tc_commit(bar(B_KVEMPTY + stage));  // every tile's P V of this stage is queued
+                    if (elect_one()) tc_commit(bar(tb + T_PVDONE + (i & 1)));
                 }
+                if (!ok) break;
+                if (elect_one()) tc_commit(bar(B_KVEMPTY + stage));  // every tile's P V of this stage is queued
             }
         }
     } else {
