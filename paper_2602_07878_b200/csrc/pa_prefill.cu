@@ -450,51 +450,56 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         auto wait_all = [&](int b_idx, uint32_t parity) -> bool {
             return __all_sync(0xffffffffu, wait(b_idx, parity));
         };
+        // This warp shares its scheduler with two softmax warps, so the loop is kept short:
+        // descriptors are the three bases below plus constants in the address field (an
+        // address inside this CTA's shared memory never carries out of its 14 bits).
+        const bool leader = elect_one();
+        const uint64_t q_desc = tc_smem_desc(sbase + OFF_Q, 16, 1024);
+        const uint64_t k_desc0 = tc_smem_desc(sbase + OFF_KV, 16, 1024);
+        const uint64_t v_desc0 = tc_smem_desc(sbase + OFF_KV + 2 * KV_HALF, KV_HALF, 1024);
         bool ok = wait_all(B_QFULL, 0);
         for (int j = 0; ok && j <= n_steps; ++j) {
             if (j < n_steps) {  // S[tile][j % 2] = Q_tile K_j^T
                 const int stage = j % ST;
                 ok = wait_all(B_KVFULL + stage, (j / ST) & 1);
                 if (!ok) break;
-                const uint32_t kb = sbase + OFF_KV + stage * STAGE_BYTES;
+                const uint64_t k_desc = k_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                const uint32_t s_col = tmem + (j & 1) * STEP;
 #pragma unroll
                 for (int t = 0; t < NT; ++t) {
-                    const int tb = C::B_TILE + 8 * t;
-                    const uint32_t qb = sbase + OFF_Q + t * Q_BYTES;
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
                         const uint64_t a =
-                            tc_smem_desc(qb + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32, 16, 1024);
-                        const uint64_t bd =
-                            tc_smem_desc(kb + (ks >> 2) * KV_HALF + (ks & 3) * 32, 16, 1024);
-                        if (elect_one())
-                            tc_mma_bf16(tmem + t * 256 + (j & 1) * STEP, a, bd, idesc_qk, ks > 0);
+                            q_desc + (uint64_t)((t * Q_BYTES + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32) >> 4);
+                        const uint64_t bd = k_desc + (uint64_t)(((ks >> 2) * KV_HALF + (ks & 3) * 32) >> 4);
+                        if (leader) tc_mma_bf16(s_col + t * 256, a, bd, idesc_qk, ks > 0);
                     }
-                    if (elect_one()) tc_commit(bar(tb + T_SFULL + (j & 1)));
+                    if (leader) tc_commit(bar(C::B_TILE + 8 * t + T_SFULL + (j & 1)));
                 }
             }
             if (j >= 1) {  // O[tile] += P_{j-1} V_{j-1}
                 const int i = j - 1, stage = i % ST;
-                const uint32_t vb = sbase + OFF_KV + stage * STAGE_BYTES + 2 * KV_HALF;
+                const uint64_t v_desc = v_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                const uint32_t p_col = tmem + (i & 1) * STEP;
 #pragma unroll
                 for (int t = 0; t < NT; ++t) {
                     const int tb = C::B_TILE + 8 * t;
                     ok = ok && wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t pt = tmem + t * 256 + (i & 1) * STEP;
 #pragma unroll
                     for (int kk = 0; kk < STEP / 16; ++kk) {
-                        // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB apart
-                        const uint64_t bd = tc_smem_desc(vb + kk * (16 * 128), KV_HALF, 1024);
-                        if (elect_one())
-                            tc_mma_bf16_ta(tmem + t * 256 + 2 * STEP, pt + kk * 8, bd, idesc_pv,
-                                           (i > 0 || kk > 0) ? 1u : 0u);
+                        // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB
+                        // apart; 16 tokens (2 KiB) per MMA
+                        const uint64_t bd = v_desc + (uint64_t)((kk * 16 * 128) >> 4);
+                        if (leader)
+                            tc_mma_bf16_ta(tmem + t * 256 + 2 * STEP, p_col + t * 256 + kk * 8, bd,
+                                           idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
                     }
-                    if (elect_one()) tc_commit(bar(tb + T_PVDONE + (i & 1)));
+                    if (leader) tc_commit(bar(tb + T_PVDONE + (i & 1)));
                 }
                 if (!ok) break;
-                if (elect_one()) tc_commit(bar(B_KVEMPTY + stage));  // every tile's P V of this stage is queued
+                if (leader) tc_commit(bar(B_KVEMPTY + stage));  // every tile's P V of this stage is queued
             }
         }
     } else {
