@@ -11,6 +11,7 @@
 #include <cstdlib>
 #include <mutex>
 #include <string>
+#include <type_traits>
 
 #include "attn_block.cuh"
 #include "internal.h"
@@ -281,6 +282,10 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 // overlap the softmax of step j.
 namespace tc {
 constexpr int ROWS = 128, STEP = 64, D = 128;
+#ifndef PAGEDKV_POLY_PAIRS
+#define PAGEDKV_POLY_PAIRS 2
+#endif
+constexpr int POLY_PAIRS = PAGEDKV_POLY_PAIRS;  // of every 8 pairs of weights, how many take the cubic
 constexpr int Q_BYTES = ROWS * D * 2;                 // two 64-dim halves of 128 rows x 128 B
 constexpr int KV_HALF = STEP * 128;                   // 64 tokens x 128 B
 constexpr int STAGE_BYTES = 4 * KV_HALF;              // K half 0, K half 1, V half 0, V half 1
@@ -441,8 +446,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         // The whole warp walks the loop and one elected lane issues: descriptor arithmetic
         // that is uniform across the warp stays off the issuing lane's critical path (issued
         // from a single-lane branch an MMA costs 50-65 cycles of issue, this way 30-40).
-        // Per step j: Q K^T of step j for every tile, then P V of step j-1 for every tile, so
-        // that the tensor pipe always has the other tile's work while one tile is in softmax.
+        // Per step j and tile: Q K^T of step j, then P V of step j-1, so that the wait for the
+        // weights comes while the tensor pipe still has the Q K^T just issued in its queue.
         // S(j % 2) is free for Q K^T of step j once P V of step j-2, which read its weights
         // from there, has been issued: MMAs of one thread execute in issue order.
         constexpr uint32_t idesc_qk = tc_idesc_bf16(ROWS, STEP, false);
@@ -459,14 +464,18 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         const uint64_t v_desc0 = tc_smem_desc(sbase + OFF_KV + 2 * KV_HALF, KV_HALF, 1024);
         bool ok = wait_all(B_QFULL, 0);
         for (int j = 0; ok && j <= n_steps; ++j) {
-            if (j < n_steps) {  // S[tile][j % 2] = Q_tile K_j^T
-                const int stage = j % ST;
+            const int stage = j % ST, pstage = (j + ST - 1) % ST;
+            if (j < n_steps) {
                 ok = wait_all(B_KVFULL + stage, (j / ST) & 1);
                 if (!ok) break;
-                const uint64_t k_desc = k_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
-                const uint32_t s_col = tmem + (j & 1) * STEP;
+            }
+            const uint64_t k_desc = k_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+            const uint64_t v_desc = v_desc0 + (uint64_t)(pstage * (STAGE_BYTES >> 4));
+            const uint32_t s_col = tmem + (j & 1) * STEP, p_col = tmem + ((j + 1) & 1) * STEP;
 #pragma unroll
-                for (int t = 0; t < NT; ++t) {
+            for (int t = 0; t < NT; ++t) {
+                const int tb = C::B_TILE + 8 * t;
+                if (j < n_steps) {  // S[t][j % 2] = Q_t K_j^T
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
                         const uint64_t a =
@@ -474,17 +483,11 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                         const uint64_t bd = k_desc + (uint64_t)(((ks >> 2) * KV_HALF + (ks & 3) * 32) >> 4);
                         if (leader) tc_mma_bf16(s_col + t * 256, a, bd, idesc_qk, ks > 0);
                     }
-                    if (leader) tc_commit(bar(C::B_TILE + 8 * t + T_SFULL + (j & 1)));
+                    if (leader) tc_commit(bar(tb + T_SFULL + (j & 1)));
                 }
-            }
-            if (j >= 1) {  // O[tile] += P_{j-1} V_{j-1}
-                const int i = j - 1, stage = i % ST;
-                const uint64_t v_desc = v_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
-                const uint32_t p_col = tmem + (i & 1) * STEP;
-#pragma unroll
-                for (int t = 0; t < NT; ++t) {
-                    const int tb = C::B_TILE + 8 * t;
-                    ok = ok && wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
+                if (j >= 1) {  // O[t] += P_{j-1} V_{j-1}; the wait falls behind the queued Q K^T
+                    const int i = j - 1;
+                    ok = wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
                     if (!ok) break;
                     tc_fence_after_sync();
 #pragma unroll
@@ -498,9 +501,10 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                     }
                     if (leader) tc_commit(bar(tb + T_PVDONE + (i & 1)));
                 }
-                if (!ok) break;
-                if (leader) tc_commit(bar(B_KVEMPTY + stage));  // every tile's P V of this stage is queued
             }
+            if (!ok) break;
+            // every tile's P V of the previous step is queued: its K/V stage may be refilled
+            if (j >= 1 && leader) tc_commit(bar(B_KVEMPTY + pstage));
         }
     } else {
         // ===================== softmax + epilogue: thread = row =====================
@@ -529,41 +533,59 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             uint32_t pk[STEP / 2];
             float corr = 1.f, lsum = 0.f;
             if (sl2 > 0.f) {
-                // fast path: maximum on the raw scores, one FMA + one EX2 per element
-                float m8[8];  // eight independent chains, then a tree
-#pragma unroll
-                for (int i = 0; i < 8; ++i) m8[i] = -INFINITY;
-                if (__any_sync(0xffffffffu, t0 + STEP - 1 > pos)) {  // diagonal step: mask
+                // fast path: maximum on the raw scores, then per pair of elements one packed
+                // FMA and either two EX2 or the packed cubic (POLY_PAIRS of every 8 pairs, so
+                // that the special-function unit and the FMA pipe share the exponentials)
+                const bool diagonal = __any_sync(0xffffffffu, t0 + STEP - 1 > pos);
+                float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (diagonal) {  // mask
 #pragma unroll
                     for (int c = 0; c < STEP; ++c) {
                         float v = __uint_as_float(sr[c >> 5][c & 31]);
                         v = (t0 + c <= pos) ? v : -INFINITY;
                         sr[c >> 5][c & 31] = __float_as_uint(v);
-                        m8[c & 7] = fmaxf(m8[c & 7], v);
+                        m4[c & 3] = fmaxf(m4[c & 3], v);
                     }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < STEP; ++c)
-                        m8[c & 7] = fmaxf(m8[c & 7], __uint_as_float(sr[c >> 5][c & 31]));
+                    for (int c = 0; c < STEP; c += 2)
+                        m4[(c >> 1) & 3] = max3(m4[(c >> 1) & 3], __uint_as_float(sr[c >> 5][c & 31]),
+                                                __uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]));
                 }
-                const float mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])),
-                                       fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7]))) * sl2;
+                const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * sl2;
                 // keep the reference maximum unless it would let a weight exceed 2^8
                 if (mx > m_ref + 8.f) {
                     corr = ex2(m_ref - mx);  // 0 on the first step
                     m_ref = mx;
                 }
                 const float nmu = m_ref == -INFINITY ? 0.f : -m_ref;
-                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint64_t sl2x2 = pack_f32x2(sl2, sl2), nmux2 = pack_f32x2(nmu, nmu);
+                uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};
+                auto weights = [&](auto use_poly) {
 #pragma unroll
-                for (int c = 0; c < STEP; c += 2) {
-                    const float e0 = ex2(fmaf(__uint_as_float(sr[c >> 5][c & 31]), sl2, nmu));
-                    const float e1 =
-                        ex2(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), sl2, nmu));
-                    ls4[(c >> 1) & 3] += e0 + e1;
-                    pk[c >> 1] = pack_bf16x2(e0, e1);
-                }
-                lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                    for (int c = 0; c < STEP; c += 2) {
+                        const uint64_t y =
+                            fma_f32x2(pack_f32x2(__uint_as_float(sr[c >> 5][c & 31]),
+                                                 __uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31])),
+                                      sl2x2, nmux2);
+                        float y0, y1, e0, e1;
+                        unpack_f32x2(y, y0, y1);
+                        if (decltype(use_poly)::value && ((c >> 1) & 7) < POLY_PAIRS) {
+                            exp2_poly_x2(pack_f32x2(fmaxf(y0, -126.f), fmaxf(y1, -126.f)), e0, e1);
+                        } else {
+                            e0 = ex2(y0);
+                            e1 = ex2(y1);
+                        }
+                        ls2[(c >> 1) & 3] = add_f32x2(ls2[(c >> 1) & 3], pack_f32x2(e0, e1));
+                        pk[c >> 1] = pack_bf16x2(e0, e1);
+                    }
+                };
+                // masked elements must come out as exact zeros: the diagonal steps keep EX2
+                if (diagonal) weights(std::false_type{}); else weights(std::true_type{});
+                float a0, a1, b0, b1;
+                unpack_f32x2(add_f32x2(ls2[0], ls2[1]), a0, a1);
+                unpack_f32x2(add_f32x2(ls2[2], ls2[3]), b0, b1);
+                lsum = (a0 + a1) + (b0 + b1);
             } else {
                 float mx = -INFINITY;
 #pragma unroll

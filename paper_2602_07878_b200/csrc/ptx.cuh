@@ -118,6 +118,50 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+// ---- packed fp32 pairs (sm_100 executes one instruction on both halves) --------------------
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// 2^y for a pair, y in [-126, 126], on the FMA pipe instead of the special-function unit:
+// y = n + f with n = round(y) (taken from the low mantissa bits of y + 1.5 * 2^23) and
+// f in [-0.5, 0.5]; 2^f by a cubic fitted to a relative error of 7.5e-5 (far below the bf16
+// rounding the weights get next); 2^n by adding n to the exponent field.
+__device__ __forceinline__ void exp2_poly_x2(uint64_t y, float& e0, float& e1) {
+    const float magic = 12582912.f;
+    const uint64_t t = add_f32x2(y, pack_f32x2(magic, magic));
+    const uint64_t n = add_f32x2(t, pack_f32x2(-magic, -magic));
+    const uint64_t f = fma_f32x2(n, pack_f32x2(-1.f, -1.f), y);
+    uint64_t p = fma_f32x2(pack_f32x2(0.0551716648f, 0.0551716648f), f,
+                           pack_f32x2(0.2426111251f, 0.2426111251f));
+    p = fma_f32x2(p, f, pack_f32x2(0.6932609677f, 0.6932609677f));
+    p = fma_f32x2(p, f, pack_f32x2(0.9999280572f, 0.9999280572f));
+    float p0, p1, t0, t1;
+    unpack_f32x2(p, p0, p1);
+    unpack_f32x2(t, t0, t1);
+    e0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+    e1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+}
+
 // two floats -> packed bf16x2 (lo in bits 0..15), round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
