@@ -462,19 +462,24 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         const uint64_t q_desc = tc_smem_desc(sbase + OFF_Q, 16, 1024);
         const uint64_t k_desc0 = tc_smem_desc(sbase + OFF_KV, 16, 1024);
         const uint64_t v_desc0 = tc_smem_desc(sbase + OFF_KV + 2 * KV_HALF, KV_HALF, 1024);
-        bool ok = wait_all(B_QFULL, 0);
+        // A barrier test is a shared-memory access that queues behind the MMAs' operand reads
+        // (150-200 cycles under load), so every barrier is tested once ahead of time and the
+        // answer is looked at only after the MMAs in between have been issued; the full wait
+        // runs only when that early test failed.
+        bool ok = wait_all(B_QFULL, 0) && wait_all(B_KVFULL, 0);
         for (int j = 0; ok && j <= n_steps; ++j) {
             const int stage = j % ST, pstage = (j + ST - 1) % ST;
-            if (j < n_steps) {
-                ok = wait_all(B_KVFULL + stage, (j / ST) & 1);
-                if (!ok) break;
-            }
+            const bool kv_next_early =
+                j + 1 < n_steps ? mbar_try_wait(bar(B_KVFULL + (j + 1) % ST), ((j + 1) / ST) & 1) : true;
             const uint64_t k_desc = k_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
             const uint64_t v_desc = v_desc0 + (uint64_t)(pstage * (STAGE_BYTES >> 4));
             const uint32_t s_col = tmem + (j & 1) * STEP, p_col = tmem + ((j + 1) & 1) * STEP;
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
                 const int tb = C::B_TILE + 8 * t;
+                const int i = j - 1;
+                const bool p_early =
+                    j >= 1 ? mbar_try_wait(bar(tb + T_PFULL + (i & 1)), (i >> 1) & 1) : true;
                 if (j < n_steps) {  // S[t][j % 2] = Q_t K_j^T
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
@@ -485,10 +490,11 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                     }
                     if (leader) tc_commit(bar(tb + T_SFULL + (j & 1)));
                 }
-                if (j >= 1) {  // O[t] += P_{j-1} V_{j-1}; the wait falls behind the queued Q K^T
-                    const int i = j - 1;
-                    ok = wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
-                    if (!ok) break;
+                if (j >= 1) {  // O[t] += P_{j-1} V_{j-1}
+                    if (!__all_sync(0xffffffffu, p_early)) {
+                        ok = wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
+                        if (!ok) break;
+                    }
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < STEP / 16; ++kk) {
@@ -505,6 +511,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             if (!ok) break;
             // every tile's P V of the previous step is queued: its K/V stage may be refilled
             if (j >= 1 && leader) tc_commit(bar(B_KVEMPTY + pstage));
+            if (j + 1 < n_steps && !__all_sync(0xffffffffu, kv_next_early))
+                ok = wait_all(B_KVFULL + (j + 1) % ST, ((j + 1) / ST) & 1);
         }
     } else {
         // ===================== softmax + epilogue: thread = row =====================
