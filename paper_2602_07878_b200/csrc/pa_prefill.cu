@@ -899,15 +899,15 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
             (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
         // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
         // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
-        const double step_us = nt == 1 ? 0.83 : 1.28;
+        const double step_us = nt == 1 ? 0.83 : 0.92;
         const int64_t s_hi = forced_split_steps ? 1 : std::min<int64_t>({cap_fit, 64, steps_bound / 8});
         for (int64_t s_try = 1; s_try <= std::max<int64_t>(1, s_hi); ++s_try) {
             int64_t T = forced_split_steps ? forced_split_steps : (steps_bound + s_try - 1) / s_try;
             const int64_t S = (steps_bound + T - 1) / T;
             if (S > cap_fit && S > 1) continue;
             const int64_t rounds = (groups * S + sm_count - 1) / sm_count;
-            double t = rounds * (T * step_us + 4.0);
-            if (S > 1) t += 6.0 + (double)total_q * H * S * (D + 2) * 4 * 2 / 2.5e6;
+            double t = rounds * (T * step_us + 10.0);
+            if (S > 1) t += 6.0 + (double)total_q * H * S * (D + 2) * 4 * 2 / 5.0e6;
             if (t < best_t) {
                 best_t = t;
                 best = {nt, S > 1 ? (int)T : 0, (int)std::max<int64_t>(S, 1)};
