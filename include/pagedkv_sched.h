@@ -64,6 +64,33 @@ typedef struct sched_step_out {
     const int64_t* finished_ids;
 } sched_step_out;
 
+/*
+ * Countermeasures (Section 7 "Countermeasures" names them without defining them; the readings
+ * taken here are stated per field).  All zero = the engine of Section 5.1 unchanged.
+ */
+#define SCHED_VICTIM_LIFO 0     /* Section 5.1.2: the most recently admitted sequence            */
+#define SCHED_VICTIM_LARGEST 1  /* fairness: the running sequence that holds the most blocks     */
+typedef struct sched_policy {
+    int32_t victim_policy;     /* SCHED_VICTIM_*                                                 */
+    int32_t demote_victims;    /* 1: a preempted sequence re-queues at the BACK of WAITING (it is
+                                  "de-escalated"), not at the front                              */
+    int32_t admit_lookahead;   /* fairness: when the head of WAITING does not fit, up to this many
+                                  requests behind it are tried (0 = strict FCFS, head-of-line
+                                  blocking as in Section 5.1.1)                                  */
+    int32_t max_output_tokens; /* quota: a request finishes after this many generated tokens even
+                                  if it asked for more (0 = no cap)                              */
+    int32_t max_seq_blocks;    /* quota: a request that would need more KV blocks than this is
+                                  finished (truncated) instead of growing (0 = no cap)           */
+} sched_policy;
+
+/* Per-request outcome in iterations (the scheduler's clock): the step it was queued at, the
+ * step that produced its first generated token (-1 if none yet), the step it finished at (-1
+ * if not yet), how often it was preempted, how many tokens it generated. */
+typedef struct sched_request_stats {
+    int64_t queued_step, first_token_step, finished_step;
+    int32_t preemptions, generated;
+} sched_request_stats;
+
 /* Returns NULL on an invalid configuration. */
 void* sched_create(const sched_config* cfg);
 void sched_destroy(void* sched);
@@ -73,6 +100,11 @@ int sched_add_request(void* sched, int64_t id, int32_t prompt_len, int32_t max_n
 /* Run one iteration.  Returns 0, or 1 when nothing is running or waiting any more. */
 int sched_step(void* sched, sched_step_out* out);
 void sched_get_stats(const void* sched, sched_stats* stats);
+/* Set the countermeasures; takes effect from the next sched_step.  Returns 0, or -1 on an
+ * unknown policy or a negative field. */
+int sched_set_policy(void* sched, const sched_policy* policy);
+/* Outcome of request `id` so far.  Returns 0, or -1 if the id is unknown. */
+int sched_get_request_stats(const void* sched, int64_t id, sched_request_stats* out);
 
 #ifdef __cplusplus
 }

@@ -8,13 +8,17 @@
 //   * recovery by swapping (the victim's blocks go to host memory and come back into newly
 //     allocated blocks) or by recomputation (its KV is dropped and prompt + generated tokens
 //     are prefilled again), prefill running in chunks under a per-iteration token budget
-//     (Appendix B.1).
+//     (Appendix B.1);
+//   * optionally the countermeasures Section 7 names (output-length and memory quotas, a
+//     fairness-aware choice of victim and of the next request to admit), as switches on the
+//     same engine so that their effect on queueing and preemption can be measured.
 // It produces, per iteration, exactly what the GPU entry points take: block tables and
 // lengths for pa_decode, slot mappings for kv_append, (query, context) lengths for
 // pa_prefill, and block-id lists for kv_swap_out / kv_swap_in.  No prompt or probe tooling.
 #include <algorithm>
 #include <cstdint>
 #include <deque>
+#include <unordered_map>
 #include <vector>
 
 #include "../../include/pagedkv_sched.h"
@@ -32,10 +36,14 @@ struct Seq {
     std::vector<int32_t> blocks;  // logical -> physical
     int32_t host_start, host_slots;  // range of host slots holding its blocks while swapped out
     int64_t admitted_at;          // order of admission, for LIFO victim choice
+    int64_t queued_step, first_token_step, finished_step;
+    int32_t preemptions;
 };
 
 struct Sched {
     sched_config cfg;
+    sched_policy policy{};
+    std::unordered_map<int64_t, int> by_id;
     std::deque<int32_t> free_blocks;
     std::vector<Seq> seqs;
     std::deque<int> waiting;  // indices into seqs, front = head of line
@@ -93,6 +101,7 @@ struct Sched {
 void preempt(Sched& S, int idx) {
     Seq& s = S.seqs[idx];
     ++S.stats.preemptions;
+    ++s.preemptions;
     int host = -1;
     if (S.cfg.preempt_mode == SCHED_PREEMPT_SWAP && s.state == DECODE)
         host = S.host_alloc((int)s.blocks.size());
@@ -113,7 +122,30 @@ void preempt(Sched& S, int idx) {
     }
     S.release(s);
     S.running.erase(std::find(S.running.begin(), S.running.end(), idx));
-    S.waiting.push_front(idx);
+    if (S.policy.demote_victims) S.waiting.push_back(idx); else S.waiting.push_front(idx);
+}
+
+// Which running sequence gives up its blocks: the last admitted one (Section 5.1.2), or, as a
+// fairness measure, the one that holds the most blocks (ties: the later admitted).
+int pick_victim(const Sched& S) {
+    if (S.policy.victim_policy == SCHED_VICTIM_LIFO) return S.running.back();
+    int best = S.running.back();
+    for (int idx : S.running)
+        if (S.seqs[idx].blocks.size() > S.seqs[best].blocks.size() ||
+            (S.seqs[idx].blocks.size() == S.seqs[best].blocks.size() &&
+             S.seqs[idx].admitted_at > S.seqs[best].admitted_at))
+            best = idx;
+    return best;
+}
+
+void finish(Sched& S, int idx) {
+    Seq& s = S.seqs[idx];
+    S.o_finished.push_back(s.id);
+    S.release(s);
+    s.state = FINISHED;
+    s.finished_step = S.stats.steps;
+    S.running.erase(std::find(S.running.begin(), S.running.end(), idx));
+    ++S.stats.finished;
 }
 
 void write_table(const Sched& S, const Seq& s, std::vector<int32_t>& dst) {
@@ -154,6 +186,10 @@ extern "C" int sched_add_request(void* sched, int64_t id, int32_t prompt_len,
     s.max_new = max_new_tokens;
     s.target = prompt_len;
     s.state = WAITING_NEW;
+    s.queued_step = S.stats.steps;
+    s.first_token_step = s.finished_step = -1;
+    if (S.by_id.count(id)) return -1;
+    S.by_id[id] = (int)S.seqs.size();
     S.seqs.push_back(s);
     S.waiting.push_back((int)S.seqs.size() - 1);
     return 0;
@@ -165,6 +201,25 @@ extern "C" void sched_get_stats(const void* sched, sched_stats* stats) {
     stats->free_blocks = (int32_t)S.free_blocks.size();
     stats->running = (int32_t)S.running.size();
     stats->waiting = (int32_t)S.waiting.size();
+}
+
+extern "C" int sched_set_policy(void* sched, const sched_policy* p) {
+    if (!sched || !p) return -1;
+    if ((p->victim_policy != SCHED_VICTIM_LIFO && p->victim_policy != SCHED_VICTIM_LARGEST) ||
+        p->admit_lookahead < 0 || p->max_output_tokens < 0 || p->max_seq_blocks < 0 ||
+        (p->demote_victims != 0 && p->demote_victims != 1))
+        return -1;
+    static_cast<Sched*>(sched)->policy = *p;
+    return 0;
+}
+
+extern "C" int sched_get_request_stats(const void* sched, int64_t id, sched_request_stats* out) {
+    const Sched& S = *static_cast<const Sched*>(sched);
+    auto it = S.by_id.find(id);
+    if (it == S.by_id.end() || !out) return -1;
+    const Seq& s = S.seqs[it->second];
+    *out = {s.queued_step, s.first_token_step, s.finished_step, s.preemptions, s.generated};
+    return 0;
 }
 
 extern "C" int sched_step(void* sched, sched_step_out* out) {
@@ -190,9 +245,14 @@ extern "C" int sched_step(void* sched, sched_step_out* out) {
             ++i;
             continue;
         }
+        // memory quota: a sequence at its cap is cut off instead of growing
+        if (S.policy.max_seq_blocks > 0 && (int)s.blocks.size() >= S.policy.max_seq_blocks) {
+            finish(S, idx);
+            continue;
+        }
         bool self_evicted = false;
         while (S.free_blocks.empty()) {
-            const int victim = S.running.back();
+            const int victim = pick_victim(S);
             preempt(S, victim);
             if (victim == idx) {
                 self_evicted = true;
@@ -209,19 +269,24 @@ extern "C" int sched_step(void* sched, sched_step_out* out) {
     for (int idx : S.running)
         if (S.seqs[idx].state == DECODE) --budget;
     bool blocked = false;
-    while (!S.waiting.empty() && (int)S.running.size() < S.cfg.max_num_seqs) {
-        const int idx = S.waiting.front();
+    size_t pos = 0;  // position in WAITING being tried; > 0 only behind a head that does not fit
+    int skipped = 0;
+    while (pos < S.waiting.size() && (int)S.running.size() < S.cfg.max_num_seqs) {
+        const int idx = S.waiting[pos];
         Seq& s = S.seqs[idx];
         const bool swapped = s.state == WAITING_SWAPPED;
         // a swapped sequence comes back whole and also needs the block of its next token
         const int need = swapped ? std::max(s.host_slots, S.blocks_for(s.len + 1))
                                  : S.blocks_for(s.target);
         if (!swapped && budget <= 0) break;  // no prefill tokens left this iteration
-        if ((int)S.free_blocks.size() < need) {  // can_allocate() fails: head-of-line blocking
-            blocked = true;
-            break;
+        if ((int)S.free_blocks.size() < need) {  // can_allocate() fails: head-of-line blocking,
+            blocked = true;                      // unless the policy lets a few requests pass
+            if (skipped >= S.policy.admit_lookahead) break;
+            ++skipped;
+            ++pos;
+            continue;
         }
-        S.waiting.pop_front();
+        S.waiting.erase(S.waiting.begin() + pos);
         S.take(s, need);
         if (swapped) {
             for (int i = 0; i < s.host_slots; ++i) {
@@ -255,7 +320,10 @@ extern "C" int sched_step(void* sched, sched_step_out* out) {
         ++s.len;
         ++s.generated;
         ++S.stats.decode_tokens;
-        if (s.generated >= s.max_new) done.push_back(idx);
+        if (s.first_token_step < 0) s.first_token_step = S.stats.steps;
+        const int cap = S.policy.max_output_tokens > 0 ? std::min(s.max_new, S.policy.max_output_tokens)
+                                                       : s.max_new;
+        if (s.generated >= cap) done.push_back(idx);
     }
     int prefill_tokens = 0;
     for (int idx : S.running) {
@@ -273,14 +341,7 @@ extern "C" int sched_step(void* sched, sched_step_out* out) {
         if (s.len == s.target) s.state = DECODE;  // decodes from the next iteration on
     }
     S.stats.prefill_tokens += prefill_tokens;
-    for (int idx : done) {
-        Seq& s = S.seqs[idx];
-        S.o_finished.push_back(s.id);
-        S.release(s);
-        s.state = FINISHED;
-        S.running.erase(std::find(S.running.begin(), S.running.end(), idx));
-        ++S.stats.finished;
-    }
+    for (int idx : done) finish(S, idx);
 
     out->n_decode = (int32_t)S.o_decode_ids.size();
     out->decode_ids = S.o_decode_ids.data();

@@ -14,6 +14,7 @@ import numpy as np
 from . import api
 
 SWAP, RECOMPUTE = 0, 1
+VICTIM_LIFO, VICTIM_LARGEST = 0, 1
 
 
 class SchedConfig(ctypes.Structure):
@@ -28,6 +29,17 @@ class SchedStats(ctypes.Structure):
                  "recomputed_tokens", "finished", "hol_blocked_steps", "decode_tokens",
                  "prefill_tokens")] + \
                [(n, ctypes.c_int32) for n in ("free_blocks", "running", "waiting", "reserved")]
+
+
+class SchedPolicy(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("victim_policy", "demote_victims", "admit_lookahead", "max_output_tokens",
+                 "max_seq_blocks")]
+
+
+class SchedRequestStats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("queued_step", "first_token_step", "finished_step")] + \
+               [(n, ctypes.c_int32) for n in ("preemptions", "generated")]
 
 
 _p64, _p32 = ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)
@@ -87,6 +99,11 @@ class Scheduler:
         L.sched_step.restype = ctypes.c_int
         L.sched_get_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(SchedStats)]
         L.sched_get_stats.restype = None
+        L.sched_set_policy.argtypes = [ctypes.c_void_p, ctypes.POINTER(SchedPolicy)]
+        L.sched_set_policy.restype = ctypes.c_int
+        L.sched_get_request_stats.argtypes = [ctypes.c_void_p, ctypes.c_int64,
+                                              ctypes.POINTER(SchedRequestStats)]
+        L.sched_get_request_stats.restype = ctypes.c_int
         self._L = L
         self.cfg = SchedConfig(num_blocks, block_size, max_num_seqs, max_batched_tokens,
                                preempt_mode, max_blocks_per_seq, host_blocks)
@@ -103,6 +120,19 @@ class Scheduler:
 
     def add_request(self, req_id: int, prompt_len: int, max_new_tokens: int) -> bool:
         return self._L.sched_add_request(self._h, req_id, prompt_len, max_new_tokens) == 0
+
+    def set_policy(self, victim_policy=VICTIM_LIFO, demote_victims=False, admit_lookahead=0,
+                   max_output_tokens=0, max_seq_blocks=0) -> None:
+        pol = SchedPolicy(victim_policy, int(demote_victims), admit_lookahead, max_output_tokens,
+                          max_seq_blocks)
+        if self._L.sched_set_policy(self._h, ctypes.byref(pol)) != 0:
+            raise ValueError("invalid scheduler policy")
+
+    def request_stats(self, req_id: int) -> SchedRequestStats:
+        r = SchedRequestStats()
+        if self._L.sched_get_request_stats(self._h, req_id, ctypes.byref(r)) != 0:
+            raise KeyError(req_id)
+        return r
 
     def stats(self) -> SchedStats:
         s = SchedStats()
