@@ -616,7 +616,8 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_spli
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pa_decode_kernel launch, from the ncu
 # capture summarised under profiles/ (None until a capture of the current kernel exists)
-NCU_TRAFFIC = {"cfg3_fullpool_mixed_gqa": 1597868584}
+NCU_TRAFFIC = {"cfg3_fullpool_mixed_gqa": 1597868584, "cfg2_llama2_7b_mha": 1099789704,
+               "cfg5_70b_gqa": 5083087816}
 
 
 def cpu_baseline(args, spec, q, k, v):
