@@ -281,28 +281,36 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 // operand reads already fill.  Two score buffers and four KV stages let Q K^T of step j+1
 // overlap the softmax of step j.
 namespace tc {
-constexpr int ROWS = 128, STEP = 64, D = 128;
+constexpr int ROWS = 128, STEP = 64;
 #ifndef PAGEDKV_POLY_PAIRS
 #define PAGEDKV_POLY_PAIRS 2
 #endif
 constexpr int POLY_PAIRS = PAGEDKV_POLY_PAIRS;  // of every 8 pairs of weights, how many take the cubic
-constexpr int Q_BYTES = ROWS * D * 2;                 // two 64-dim halves of 128 rows x 128 B
-constexpr int KV_HALF = STEP * 128;                   // 64 tokens x 128 B
-constexpr int STAGE_BYTES = 4 * KV_HALF;              // K half 0, K half 1, V half 0, V half 1
-// NT = row tiles per CTA (two tiles = two softmax warpgroups taking turns on the tensor pipe
-// and sharing the KV stages).
-template <int NT>
+constexpr int GROUP_BYTES = STEP * 128;  // one 64-dim column group of a 64-token K or V tile
+// D = head_dim (64, 128, 256); NT = row tiles per CTA (two tiles = two softmax warpgroups
+// taking turns on the tensor pipe and sharing the K/V rings).
+template <int D, int NT>
 struct Cfg {
-    static constexpr int ST = 4;
-    static constexpr int OFF_Q = 0, OFF_KV = NT * Q_BYTES;
-    static constexpr int OFF_BAR = OFF_KV + ST * STAGE_BYTES;
+    static constexpr int NG = D / 64;                     // 64-dim column groups
+    static constexpr int Q_GROUP = ROWS * 128;            // one column group of a Q tile
+    static constexpr int Q_BYTES = NG * Q_GROUP;
+    static constexpr int TILE_BYTES = NG * GROUP_BYTES;   // K (or V) of one 64-token step
+    // K is free again once Q K^T of its step has run, V only after P V: separate rings, and
+    // at head_dim 256 (64 KB of Q, 32 KB per tile) the V ring is the deeper one
+    static constexpr int KS = D == 256 ? 2 : 4, VS = D == 256 ? 3 : 4;
+    static constexpr int OFF_Q = 0, OFF_K = NT * Q_BYTES, OFF_V = OFF_K + KS * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_V + VS * TILE_BYTES;
     // barriers (8 bytes each): shared ones, then eight per tile
-    static constexpr int B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + ST, B_TILE = B_KVEMPTY + ST;
+    static constexpr int B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + KS, B_VFULL = B_KEMPTY + KS,
+                         B_VEMPTY = B_VFULL + VS, B_TILE = B_VEMPTY + VS;
     static constexpr int B_COUNT = B_TILE + 8 * NT;
     static constexpr int OFF_MISC = OFF_BAR + B_COUNT * 8;  // tmem base, abort flag, bad flag
     static constexpr int SMEM_BYTES = OFF_MISC + 64 + 1024;  // + slack for 1024-byte alignment
-    // per tile: S0 [0,64) S1 [64,128) O [128,256); P of step j lies over S(j % 2) [0,32)
-    static constexpr int TMEM_COLS = 256 * NT;
+    // per tile: S0 [0,64) S1 [64,128) O [128,128+D); P of step j lies over S(j % 2) [0,32)
+    static constexpr int TILE_COLS = 2 * STEP + D;
+    static constexpr int TMEM_COLS = NT * TILE_COLS <= 256 ? 256 : 512;
+    static_assert(NT * TILE_COLS <= 512, "tensor memory holds 512 columns");
+    static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
     static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + 1, THREADS = (4 * NT + 2) * 32;
 };
 // per-tile barrier indices, relative to Cfg::B_TILE + 8 * tile
@@ -311,7 +319,7 @@ enum { T_SFULL = 0, T_PFULL = 2, T_PVDONE = 4 };
 
 struct PrefillTcParams {
     PrefillParams base;
-    int tokens_per_tile;  // 128 / G
+    int tokens_per_tile;  // 128 / G, rounded down: rows tokens_per_tile * G .. 127 of a tile are idle
     // KV split: a unit covers `split_steps` 64-token steps of its tile's visible context (0 =
     // all of it).  A sequence with more than one split leaves, per (query row, split), an
     // un-normalised fp32 output row in part_o[(row * split_cap + s) * D] and its reference
@@ -322,16 +330,19 @@ struct PrefillTcParams {
     float* part_o;
 };
 
-template <int NT>
-__global__ void __launch_bounds__(tc::Cfg<NT>::THREADS, 1)
+template <int D, int NT>
+__global__ void __launch_bounds__(tc::Cfg<D, NT>::THREADS, 1)
 pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                      const __grid_constant__ CUtensorMap kmap,
                      const __grid_constant__ CUtensorMap vmap, const PrefillTcParams tp) {
     using namespace tc;
-    using C = Cfg<NT>;
-    constexpr int ST = C::ST, OFF_Q = C::OFF_Q, OFF_KV = C::OFF_KV;
+    using C = Cfg<D, NT>;
+    constexpr int NG = C::NG, KS = C::KS, VS = C::VS, Q_BYTES = C::Q_BYTES, TILE_BYTES = C::TILE_BYTES;
+    constexpr int OFF_Q = C::OFF_Q, OFF_K = C::OFF_K, OFF_V = C::OFF_V;
     constexpr int OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC, TMEM_COLS = C::TMEM_COLS;
-    constexpr int B_QFULL = C::B_QFULL, B_KVFULL = C::B_KVFULL, B_KVEMPTY = C::B_KVEMPTY;
+    constexpr int TILE_COLS = C::TILE_COLS;
+    constexpr int B_QFULL = C::B_QFULL, B_KFULL = C::B_KFULL, B_KEMPTY = C::B_KEMPTY;
+    constexpr int B_VFULL = C::B_VFULL, B_VEMPTY = C::B_VEMPTY;
     const PrefillParams& p = tp.base;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -367,10 +378,12 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     const int n_steps = min(pos_max / STEP + 1 - j0, n_split > 1 ? tp.split_steps : 0x7fffffff);
     if (n_steps <= 0) return;                           // the tile sees nothing of this split
     const int nblk_seq = (L + BS - 1) / BS;
+    const int rows_used = tpt * G;                      // < 128 when G does not divide 128
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
-        for (int i = 0; i < ST; ++i) mbar_init(bar(B_KVFULL + i), 1), mbar_init(bar(B_KVEMPTY + i), 1);
+        for (int i = 0; i < KS; ++i) mbar_init(bar(B_KFULL + i), 1), mbar_init(bar(B_KEMPTY + i), 1);
+        for (int i = 0; i < VS; ++i) mbar_init(bar(B_VFULL + i), 1), mbar_init(bar(B_VEMPTY + i), 1);
         for (int t = 0; t < NT; ++t)
             for (int i = 0; i < 2; ++i) {
                 mbar_init(bar(C::B_TILE + 8 * t + T_SFULL + i), 1);
@@ -380,6 +393,18 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         mbar_init_fence();
         misc[1] = 0;
         misc[2] = 0;
+    }
+    // rows of the Q tiles that no (token, head) pair maps to are never loaded: give them zeros
+    if (rows_used < ROWS && warp < 4 * NT) {
+        const int ti = warp >> 2, row = (warp & 3) * 32 + lane;
+        if (row >= rows_used)
+            for (int g = 0; g < NG; ++g)
+                for (int c = 0; c < 8; ++c)
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(
+                                     sbase + OFF_Q + ti * Q_BYTES + g * C::Q_GROUP + row * 128 + c * 16),
+                                 "r"(0u)
+                                 : "memory");
+        fence_proxy_async_smem();
     }
     if (warp == C::MMA_WARP) tmem_alloc(sbase + OFF_MISC, TMEM_COLS);
     tc_fence_before_sync();
@@ -403,43 +428,47 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             tma_prefetch_desc(&qmap);
             tma_prefetch_desc(&kmap);
             tma_prefetch_desc(&vmap);
-            mbar_arrive_expect_tx(bar(B_QFULL), NT * Q_BYTES);
-            for (int t = 0; t < NT; ++t) {  // tile t holds query tokens tok0 + t * tpt ..
-                const uint32_t qd = sbase + OFF_Q + t * Q_BYTES;
-                tma_load_4d(qd, &qmap, bar(B_QFULL), 0, 0, kvh, q0 + tok0 + t * tpt);
-                tma_load_4d(qd + Q_BYTES / 2, &qmap, bar(B_QFULL), 64, 0, kvh, q0 + tok0 + t * tpt);
-            }
+            mbar_arrive_expect_tx(bar(B_QFULL), NT * NG * rows_used * 128);
+            for (int t = 0; t < NT; ++t)  // tile t holds query tokens tok0 + t * tpt ..
+                for (int g = 0; g < NG; ++g)
+                    tma_load_4d(sbase + OFF_Q + t * Q_BYTES + g * C::Q_GROUP, &qmap, bar(B_QFULL),
+                                g * 64, 0, kvh, q0 + tok0 + t * tpt);
         }
         const int32_t* table = p.block_tables + (size_t)b * p.max_blocks;
         // block ids are fetched 32 at a time, one window ahead; the unit starts at block 4 * j0
         const int win0 = (j0 * 4) & ~31;
         int ids = win0 + lane < nblk_seq ? __ldg(&table[win0 + lane]) : p.NB;
         int ids_next = win0 + 32 + lane < nblk_seq ? __ldg(&table[win0 + 32 + lane]) : p.NB;
+        // lane l < 4 * NG: block l / NG of the step, column group l % NG
+        const int blk = lane / NG, grp = lane - blk * NG;
+        const uint32_t tile_off = grp * GROUP_BYTES + blk * (BS * 128);
         for (int j = 0; j < n_steps; ++j) {
-            const int stage = j % ST;
-            if (j >= ST && !wait(B_KVEMPTY + stage, ((j / ST) - 1) & 1)) break;
             const int blk0 = (j0 + j) * 4;
             if (blk0 > win0 && (blk0 & 31) == 0) {
                 ids = ids_next;
                 ids_next = blk0 + 32 + lane < nblk_seq ? __ldg(&table[blk0 + 32 + lane]) : p.NB;
             }
-            // lane l < 16: block l>>2 of the step, tile l&3 (K half 0/1, V half 0/1)
-            const int id = __shfl_sync(0xffffffffu, ids, (blk0 + (lane >> 2)) & 31);
-            const bool used = blk0 + (lane >> 2) < nblk_seq;
-            if (used && (unsigned)id >= (unsigned)p.NB && (lane & 3) == 0) {
+            const int id = __shfl_sync(0xffffffffu, ids, (blk0 + (blk & 3)) & 31);
+            const bool used = blk0 + blk < nblk_seq;
+            if (lane < 4 * NG && used && (unsigned)id >= (unsigned)p.NB && grp == 0) {
                 misc[2] = 1;
                 atomicOr(p.status, PA_STATUS_BAD_BLOCK_ID);
             }
-            if (lane == 0) mbar_arrive_expect_tx(bar(B_KVFULL + stage), STAGE_BYTES);
+            // an id outside the pool is out of the tensor's bounds and reads as zeros
+            const int coord = used ? id : p.NB;
+            const int ks = j % KS, vs = j % VS;
+            if (j >= KS && !wait(B_KEMPTY + ks, ((j / KS) - 1) & 1)) break;
+            if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), TILE_BYTES);
             __syncwarp();
-            if (lane < 16) {
-                const int which = lane & 3;
-                const uint32_t dst = sbase + OFF_KV + stage * STAGE_BYTES + which * KV_HALF +
-                                     (lane >> 2) * (BS * 128);
-                // an id outside the pool is out of the tensor's bounds and reads as zeros
-                tma_load_4d(dst, which < 2 ? &kmap : &vmap, bar(B_KVFULL + stage), (which & 1) * 64,
-                            0, kvh, used ? id : p.NB);
-            }
+            if (lane < 4 * NG)
+                tma_load_4d(sbase + OFF_K + ks * TILE_BYTES + tile_off, &kmap, bar(B_KFULL + ks),
+                            grp * 64, 0, kvh, coord);
+            if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
+            if (lane == 0) mbar_arrive_expect_tx(bar(B_VFULL + vs), TILE_BYTES);
+            __syncwarp();
+            if (lane < 4 * NG)
+                tma_load_4d(sbase + OFF_V + vs * TILE_BYTES + tile_off, &vmap, bar(B_VFULL + vs),
+                            grp * 64, 0, kvh, coord);
         }
     } else if (warp == C::MMA_WARP) {
         // ===================== MMA issuer =====================
@@ -460,37 +489,44 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         // address inside this CTA's shared memory never carries out of its 14 bits).
         const bool leader = elect_one();
         const uint64_t q_desc = tc_smem_desc(sbase + OFF_Q, 16, 1024);
-        const uint64_t k_desc0 = tc_smem_desc(sbase + OFF_KV, 16, 1024);
-        const uint64_t v_desc0 = tc_smem_desc(sbase + OFF_KV + 2 * KV_HALF, KV_HALF, 1024);
+        const uint64_t k_desc0 = tc_smem_desc(sbase + OFF_K, 16, 1024);
+        const uint64_t v_desc0 = tc_smem_desc(sbase + OFF_V, GROUP_BYTES, 1024);
         // A barrier test is a shared-memory access that queues behind the MMAs' operand reads
         // (150-200 cycles under load), so every barrier is tested once ahead of time and the
         // answer is looked at only after the MMAs in between have been issued; the full wait
         // runs only when that early test failed.
-        bool ok = wait_all(B_QFULL, 0) && wait_all(B_KVFULL, 0);
+        bool ok = wait_all(B_QFULL, 0) && wait_all(B_KFULL, 0);
         for (int j = 0; ok && j <= n_steps; ++j) {
-            const int stage = j % ST, pstage = (j + ST - 1) % ST;
-            const bool kv_next_early =
-                j + 1 < n_steps ? mbar_try_wait(bar(B_KVFULL + (j + 1) % ST), ((j + 1) / ST) & 1) : true;
-            const uint64_t k_desc = k_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
-            const uint64_t v_desc = v_desc0 + (uint64_t)(pstage * (STAGE_BYTES >> 4));
+            const int i = j - 1;  // the step whose P V is issued in this iteration
+            const int ks = j % KS, vs = (j + VS - 1) % VS;
+            const bool k_next_early =
+                j + 1 < n_steps ? mbar_try_wait(bar(B_KFULL + (j + 1) % KS), ((j + 1) / KS) & 1) : true;
+            const bool v_early = j >= 1 ? mbar_try_wait(bar(B_VFULL + vs), (i / VS) & 1) : true;
+            const uint64_t k_desc = k_desc0 + (uint64_t)(ks * (TILE_BYTES >> 4));
+            const uint64_t v_desc = v_desc0 + (uint64_t)(vs * (TILE_BYTES >> 4));
             const uint32_t s_col = tmem + (j & 1) * STEP, p_col = tmem + ((j + 1) & 1) * STEP;
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
                 const int tb = C::B_TILE + 8 * t;
-                const int i = j - 1;
                 const bool p_early =
                     j >= 1 ? mbar_try_wait(bar(tb + T_PFULL + (i & 1)), (i >> 1) & 1) : true;
                 if (j < n_steps) {  // S[t][j % 2] = Q_t K_j^T
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
+                    for (int kk = 0; kk < D / 16; ++kk) {
                         const uint64_t a =
-                            q_desc + (uint64_t)((t * Q_BYTES + (ks >> 2) * (Q_BYTES / 2) + (ks & 3) * 32) >> 4);
-                        const uint64_t bd = k_desc + (uint64_t)(((ks >> 2) * KV_HALF + (ks & 3) * 32) >> 4);
-                        if (leader) tc_mma_bf16(s_col + t * 256, a, bd, idesc_qk, ks > 0);
+                            q_desc + (uint64_t)((t * Q_BYTES + (kk >> 2) * C::Q_GROUP + (kk & 3) * 32) >> 4);
+                        const uint64_t bd = k_desc + (uint64_t)(((kk >> 2) * GROUP_BYTES + (kk & 3) * 32) >> 4);
+                        if (leader) tc_mma_bf16(s_col + t * TILE_COLS, a, bd, idesc_qk, kk > 0);
                     }
                     if (leader) tc_commit(bar(tb + T_SFULL + (j & 1)));
+                    // the last tile's Q K^T was the last reader of this step's K
+                    if (t == NT - 1 && leader) tc_commit(bar(B_KEMPTY + ks));
                 }
                 if (j >= 1) {  // O[t] += P_{j-1} V_{j-1}
+                    if (t == 0 && !__all_sync(0xffffffffu, v_early)) {
+                        ok = wait_all(B_VFULL + vs, (i / VS) & 1);
+                        if (!ok) break;
+                    }
                     if (!__all_sync(0xffffffffu, p_early)) {
                         ok = wait_all(tb + T_PFULL + (i & 1), (i >> 1) & 1);
                         if (!ok) break;
@@ -498,21 +534,21 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < STEP / 16; ++kk) {
-                        // V is MN-major: 64-dim column groups KV_HALF apart, 8-token groups 1 KiB
-                        // apart; 16 tokens (2 KiB) per MMA
+                        // V is MN-major: 64-dim column groups GROUP_BYTES apart, 8-token groups
+                        // 1 KiB apart; 16 tokens (2 KiB) per MMA
                         const uint64_t bd = v_desc + (uint64_t)((kk * 16 * 128) >> 4);
                         if (leader)
-                            tc_mma_bf16_ta(tmem + t * 256 + 2 * STEP, p_col + t * 256 + kk * 8, bd,
-                                           idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+                            tc_mma_bf16_ta(tmem + t * TILE_COLS + 2 * STEP, p_col + t * TILE_COLS + kk * 8,
+                                           bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
                     }
                     if (leader) tc_commit(bar(tb + T_PVDONE + (i & 1)));
                 }
             }
             if (!ok) break;
-            // every tile's P V of the previous step is queued: its K/V stage may be refilled
-            if (j >= 1 && leader) tc_commit(bar(B_KVEMPTY + pstage));
-            if (j + 1 < n_steps && !__all_sync(0xffffffffu, kv_next_early))
-                ok = wait_all(B_KVFULL + (j + 1) % ST, ((j + 1) / ST) & 1);
+            // every tile's P V of the previous step is queued: its V tile may be refilled
+            if (j >= 1 && leader) tc_commit(bar(B_VEMPTY + vs));
+            if (j + 1 < n_steps && !__all_sync(0xffffffffu, k_next_early))
+                ok = wait_all(B_KFULL + (j + 1) % KS, ((j + 1) / KS) & 1);
         }
     } else {
         // ===================== softmax + epilogue: thread = row =====================
@@ -520,10 +556,10 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         const int row = (warp & 3) * 32 + lane;
         const int tk = row / G, hd = row - tk * G;
         const int qtok = tok0 + ti * tpt + tk;          // query token within the sequence's chunk
-        const bool row_ok = qtok < ql;
+        const bool row_ok = row < rows_used && qtok < ql;  // idle rows exist when G does not divide 128
         const int pos = row_ok ? L - ql + qtok : 0x7fffffff;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tcol = tmem + ti * 256;          // this tile's S0, S1, O columns
+        const uint32_t tcol = tmem + ti * TILE_COLS;    // this tile's S0, S1, O columns
         const int tb = C::B_TILE + 8 * ti;              // this tile's barriers
         const float sl2 = p.scale_log2;
         float m_ref = -INFINITY, l = 0.f;
@@ -639,15 +675,15 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             bool zeroed = false;
             // slots past the end of the sequence may hold anything: zero their V rows
             if (ti == 0 && t0 + STEP > L) {  // one warpgroup does it; P V of every tile follows its p_full
-                ok = wait(B_KVFULL + (j % ST), (j / ST) & 1);
+                ok = wait(B_VFULL + (j % VS), (j / VS) & 1);
                 if (!ok) break;
                 const int r0 = max(0, L - t0);                      // first unused row of the step
                 const int r1 = min(STEP, ((L + BS - 1) / BS) * BS - t0);  // end of the partial block
-                const uint32_t vb = sbase + OFF_KV + (j % ST) * STAGE_BYTES + 2 * KV_HALF;
-                for (int e = row; e < (r1 - r0) * 16; e += 128) {
-                    const int r = r0 + (e >> 4), c = e & 15;  // 16 chunks: 8 per half
+                const uint32_t vb = sbase + OFF_V + (j % VS) * TILE_BYTES;
+                for (int e = row; e < (r1 - r0) * (D / 8); e += 128) {
+                    const int r = r0 + e / (D / 8), c = e % (D / 8);  // 16-byte chunks, 8 per group
                     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(
-                                     vb + (c >> 3) * KV_HALF + r * 128 + (c & 7) * 16),
+                                     vb + (c >> 3) * GROUP_BYTES + r * 128 + (c & 7) * 16),
                                  "r"(0u)
                                  : "memory");
                 }
@@ -728,8 +764,9 @@ struct PrefillMergeParams {
 //   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,   M = max_s m_s
 // over the splits the row's tile has visited.  Rows of sequences with a single split were
 // written by the attention kernel itself and are skipped, as are rows of refused sequences.
+template <int D>
 __global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMergeParams p) {
-    constexpr int D = 128;
+    constexpr int NV = (D / 4 + 31) / 32;  // float4 pieces of a row per lane
     pdl_launch_dependents();
     pdl_wait();
     const int lane = threadIdx.x & 31;
@@ -764,29 +801,44 @@ __global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMerg
     for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     bad = __any_sync(0xffffffffu, bad);
     const float4* po = reinterpret_cast<const float4*>(p.part_o) + (size_t)row * p.split_cap * (D / 4);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     float lsum = 0.f;
 #pragma unroll 4
     for (int s = 0; s < n_vis; ++s) {
-        const float2 v = ml[s];
-        const float4 o = po[(size_t)s * (D / 4) + lane];
-        const float w = v.x == -INFINITY ? 0.f : ex2(v.x - M);
-        acc.x = fmaf(w, o.x, acc.x);
-        acc.y = fmaf(w, o.y, acc.y);
-        acc.z = fmaf(w, o.z, acc.z);
-        acc.w = fmaf(w, o.w, acc.w);
-        lsum = fmaf(w, v.y, lsum);
+        const float2 v2 = ml[s];
+        const float w = v2.x == -INFINITY ? 0.f : ex2(v2.x - M);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c = lane + 32 * v;
+            if (c < D / 4) {
+                const float4 o = po[(size_t)s * (D / 4) + c];
+                acc[v].x = fmaf(w, o.x, acc[v].x);
+                acc[v].y = fmaf(w, o.y, acc[v].y);
+                acc[v].z = fmaf(w, o.z, acc[v].z);
+                acc[v].w = fmaf(w, o.w, acc[v].w);
+            }
+        }
+        lsum = fmaf(w, v2.y, lsum);
     }
     const float inv = (bad || !(lsum > 0.f)) ? 0.f : 1.f / lsum;
-    uint2 w;
-    w.x = pack_bf16x2(acc.x * inv, acc.y * inv);
-    w.y = pack_bf16x2(acc.z * inv, acc.w * inv);
-    if (bad) w = make_uint2(0u, 0u);
-    reinterpret_cast<uint2*>(p.out + (size_t)row * D)[lane] = w;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c = lane + 32 * v;
+        if (c < D / 4) {
+            uint2 w;
+            w.x = bad ? 0u : pack_bf16x2(acc[v].x * inv, acc[v].y * inv);
+            w.y = bad ? 0u : pack_bf16x2(acc[v].z * inv, acc[v].w * inv);
+            reinterpret_cast<uint2*>(p.out + (size_t)row * D)[c] = w;
+        }
+    }
 }
 
-// tensor map over the packed queries viewed as [total_q][Hkv][G][D]: box 64 x G x 1 x (128/G)
-static int make_q_map(CUtensorMap* map, const void* q, int total_q, int Hkv, int G, int D) {
+// tensor map over the packed queries viewed as [total_q][Hkv][G][D]: box 64 x G x 1 x tokens
+// per tile (one 64-dim column group of a row tile per copy)
+static int make_q_map(CUtensorMap* map, const void* q, int total_q, int Hkv, int G, int D,
+                      int tokens_per_tile) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -806,7 +858,7 @@ static int make_q_map(CUtensorMap* map, const void* q, int total_q, int Hkv, int
     }
     cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)G, (cuuint64_t)Hkv, (cuuint64_t)total_q};
     cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)G * D * 2, (cuuint64_t)Hkv * G * D * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)G, 1, (cuuint32_t)(128 / G)};
+    cuuint32_t box[4] = {64, (cuuint32_t)G, 1, (cuuint32_t)tokens_per_tile};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides,
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -818,17 +870,17 @@ static int make_q_map(CUtensorMap* map, const void* q, int total_q, int Hkv, int
     return PA_OK;
 }
 
-template <int NT>
+template <int D, int NT>
 static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
                              const PrefillTcParams& tp, int max_ctas, const DeviceInfo& dev,
                              cudaStream_t st) {
-    using C = tc::Cfg<NT>;
+    using C = tc::Cfg<D, NT>;
     static int configured_dev = -1;
     static std::mutex mu;
     {
         std::lock_guard<std::mutex> lk(mu);
         if (configured_dev != dev.device) {
-            int rc = check_cuda(cudaFuncSetAttribute(pa_prefill_tc_kernel<NT>,
+            int rc = check_cuda(cudaFuncSetAttribute(pa_prefill_tc_kernel<D, NT>,
                                                      cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      C::SMEM_BYTES));
             if (rc) return rc;
@@ -846,7 +898,7 @@ static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     count_launch();
-    return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_tc_kernel<NT>, qm, km, vm, tp));
+    return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_tc_kernel<D, NT>, qm, km, vm, tp));
 }
 
 }  // namespace pk
@@ -892,14 +944,15 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
     const int tpt = 128 / G;
     TcShape best = {1, 0, 1};
     double best_t = 1e30;
-    for (int nt = 1; nt <= 2; ++nt) {
-        if (forced_tiles && nt != forced_tiles) continue;
+    for (int nt = 1; nt <= (D == 256 ? 1 : 2); ++nt) {  // head_dim 256: one tile fills the TMEM
+        if (forced_tiles && nt != forced_tiles && D != 256) continue;
         const int64_t tpg = (int64_t)nt * tpt;
         const int64_t groups =
             (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
         // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
         // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
-        const double step_us = nt == 1 ? 0.83 : 0.92;
+        // (head_dim 128; the other head dims scale the tensor work of a step)
+        const double step_us = (nt == 1 ? 0.83 : 0.92) * (D == 256 ? 1.6 : D == 64 ? 0.8 : 1.0);
         const int64_t s_hi = forced_split_steps ? 1 : std::min<int64_t>({cap_fit, 64, steps_bound / 8});
         for (int64_t s_try = 1; s_try <= std::max<int64_t>(1, s_hi); ++s_try) {
             int64_t T = forced_split_steps ? forced_split_steps : (steps_bound + s_try - 1) / s_try;
@@ -967,12 +1020,12 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
     plan.batch = batch;
     plan.max_blocks = max_blocks_per_seq;
     plan.total_q = total_q;
-    // tensor-core path: 128-row tiles; needs head_dim 128 and a group size that divides 128
+    // tensor-core path: 128-row tiles of (token, head) pairs of one KV-head group
     static const bool force_mma = [] {
         const char* e = std::getenv("PAGEDKV_PREFILL");
         return e && std::string(e) == "mma";
     }();
-    const bool use_tc = !force_mma && D == 128 && (128 % G) == 0;
+    const bool use_tc = !force_mma && (D == 64 || D == 128 || D == 256) && G <= 128;
     static const int forced_tiles = [] {
         const char* e = std::getenv("PAGEDKV_PREFILL_TILES");
         const int v = e ? std::atoi(e) : 0;
@@ -997,7 +1050,7 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
                                  dev.sm_count, cap_fit, forced_tiles, forced_steps);
     }
     g_last_shape = use_tc ? ts : TcShape{0, 0, 1};
-    plan.tpg = use_tc ? ts.tiles_per_cta * (128 / G) : 16 / G;
+    plan.tpg = use_tc ? ts.tiles_per_cta * (128 / G) : 16 / G;  // 128 / G rounds down
     plan.split_steps = ts.split_steps;
     plan.hdr = hdr;
     plan.gstart = hdr + PF_WORDS;
@@ -1026,7 +1079,7 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
     pp.scale_log2 = scale * 1.4426950408889634f;
     if (use_tc) {
         CUtensorMap qm;
-        rc = make_q_map(&qm, q, total_q, pp.Hkv, G, D);
+        rc = make_q_map(&qm, q, total_q, pp.Hkv, G, D, 128 / G);
         if (rc) return rc;
         PrefillTcParams tp;
         tp.base = pp;
@@ -1037,8 +1090,12 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
         tp.part_o = tp.part_ml + (size_t)total_q * H * ts.split_cap * 2;
         const int64_t max_ctas = ((int64_t)total_q / plan.tpg + batch) * pp.Hkv * ts.split_cap;
         if (max_ctas > INT32_MAX) return PA_ERR_ARG;
-        rc = ts.tiles_per_cta == 2 ? launch_prefill_tc<2>(qm, km, vm, tp, (int)max_ctas, dev, st)
-                                   : launch_prefill_tc<1>(qm, km, vm, tp, (int)max_ctas, dev, st);
+        const bool two = ts.tiles_per_cta == 2;
+        rc = D == 256  ? launch_prefill_tc<256, 1>(qm, km, vm, tp, (int)max_ctas, dev, st)
+             : D == 128 ? (two ? launch_prefill_tc<128, 2>(qm, km, vm, tp, (int)max_ctas, dev, st)
+                               : launch_prefill_tc<128, 1>(qm, km, vm, tp, (int)max_ctas, dev, st))
+                        : (two ? launch_prefill_tc<64, 2>(qm, km, vm, tp, (int)max_ctas, dev, st)
+                               : launch_prefill_tc<64, 1>(qm, km, vm, tp, (int)max_ctas, dev, st));
         if (rc || ts.split_steps == 0) return rc;
         PrefillMergeParams mp;
         mp.ctx_lens = ctx_lens;
@@ -1063,7 +1120,9 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         count_launch();
-        return check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel, mp));
+        return check_cuda(D == 256   ? cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel<256>, mp)
+                          : D == 128 ? cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel<128>, mp)
+                                     : cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel<64>, mp));
     }
     return D == 256   ? launch_prefill<256>(km, vm, pp, dev, st)
            : D == 128 ? launch_prefill<128>(km, vm, pp, dev, st)

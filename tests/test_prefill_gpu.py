@@ -60,7 +60,35 @@ def test_mixed_chunks_match_oracle(H, Hkv, D):
     out = torch_to_f64(g.run(spec.seq_lens, cu))
     ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
     assert int(g.status.item()) == 0
+    assert api.pa_prefill_last_launch()[0] in (1, 2)   # every supported shape runs on tcgen05
     assert_parity(out, ref, f"H{H}/{Hkv} D{D}")
+
+
+def test_warp_mma_kernel_in_a_child_process():
+    # PAGEDKV_PREFILL=mma (read once per process) selects the warp-level MMA kernel
+    import os, subprocess, sys, textwrap
+    code = textwrap.dedent("""
+        import sys
+        sys.path.insert(0, "tests")
+        import numpy as np, torch
+        import oracle
+        from paper_2602_07878_b200 import api
+        from test_prefill_gpu import GpuPrefill, make_case
+        from helpers import assert_parity, torch_to_f64
+        for H, Hkv, D in [(8, 2, 128), (6, 2, 64), (16, 8, 256)]:
+            spec, q, k, v, cu = make_case([37, 64, 5, 130, 1, 700], [37, 10, 0, 33, 1, 300], H, Hkv, D, seed=3)
+            g = GpuPrefill(spec, q, k, v)
+            out = torch_to_f64(g.run(spec.seq_lens, cu))
+            assert api.pa_prefill_last_launch()[0] == 0
+            ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+            assert int(g.status.item()) == 0
+            assert_parity(out, ref, f"warp MMA H{H}/{Hkv} D{D}")
+        print("child ok")
+    """)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True,
+                         env=dict(os.environ, PAGEDKV_PREFILL="mma"), timeout=600)
+    assert res.returncode == 0 and "child ok" in res.stdout, res.stdout + res.stderr
 
 
 def test_single_query_token_equals_decode_bits():
@@ -143,6 +171,23 @@ def test_large_chunk_takes_the_two_tile_kernel():
 
 
 # ---- KV range split over CTAs (pa_prefill_split) --------------------------------------------
+
+@pytest.mark.parametrize("H,Hkv,D", [(8, 8, 64), (6, 2, 64), (10, 2, 128), (16, 8, 256), (4, 1, 256)])
+def test_kv_split_other_head_dims_and_group_sizes(H, Hkv, D):
+    # head_dim 64 and 256, and group sizes that do not divide 128 (idle rows in every tile)
+    ctx = [2999, 130, 1031, 64]
+    qlens = [300, 130, 7, 1]
+    spec, q, k, v, cu = make_case(ctx, qlens, H, Hkv, D, seed=90 + H + D)
+    split = 512
+    max_splits = -(-spec.block_tables.shape[1] * 16 // split)
+    g = GpuPrefill(spec, q, k, v, max_splits=max_splits)
+    out = torch_to_f64(g.run(spec.seq_lens, cu, split=split))
+    tiles, tok, cap = api.pa_prefill_last_launch()
+    assert tiles == (1 if D == 256 else tiles) and tiles in (1, 2) and tok == split and cap == max_splits
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, f"H{H}/{Hkv} D{D} split")
+
 
 @pytest.mark.parametrize("H,Hkv", [(4, 4), (32, 8), (16, 1)])
 @pytest.mark.parametrize("split", [64, 192, 1024])
