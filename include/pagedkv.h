@@ -266,8 +266,7 @@ int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const 
  *   workspace         dev, 256-byte aligned, >= pa_prefill_workspace_bytes(batch); splits are
  *                     used up to what pa_prefill_split_workspace_bytes(shape, batch, total_q,
  *                     splits) says fits.
- * Splitting needs head_dim 128 and a group size H / Hkv that divides 128 (the tensor-core
- * kernel); other shapes run unsplit.  pa_prefill is this call with kv_split_tokens = 0.
+ * pa_prefill is this call with kv_split_tokens = 0.
  * Two or three kernels are enqueued.  Errors as for pa_prefill; a split that met a bad
  * block id zeroes the rows that depend on it.
  */

@@ -295,9 +295,13 @@ struct Cfg {
     static constexpr int Q_GROUP = ROWS * 128;            // one column group of a Q tile
     static constexpr int Q_BYTES = NG * Q_GROUP;
     static constexpr int TILE_BYTES = NG * GROUP_BYTES;   // K (or V) of one 64-token step
-    // K is free again once Q K^T of its step has run, V only after P V: separate rings, and
-    // at head_dim 256 (64 KB of Q, 32 KB per tile) the V ring is the deeper one
-    static constexpr int KS = D == 256 ? 2 : 4, VS = D == 256 ? 3 : 4;
+    // Head_dim 64 and 128: four stages, K and V of a step signalled and released together
+    // (one barrier test and one commit less per step for the MMA warp).  Head_dim 256 (64 KB
+    // of Q, 32 KB per tile) has room for five tiles only: K, free again once Q K^T of its
+    // step has run, gets two, V, needed until P V, gets three (measured: the other way round
+    // is 1.6 times slower), each ring with its own barriers.
+    static constexpr bool SPLIT_RINGS = D == 256;
+    static constexpr int KS = SPLIT_RINGS ? 2 : 4, VS = SPLIT_RINGS ? 3 : 4;
     static constexpr int OFF_Q = 0, OFF_K = NT * Q_BYTES, OFF_V = OFF_K + KS * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + VS * TILE_BYTES;
     // barriers (8 bytes each): shared ones, then eight per tile
@@ -342,7 +346,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     constexpr int OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC, TMEM_COLS = C::TMEM_COLS;
     constexpr int TILE_COLS = C::TILE_COLS;
     constexpr int B_QFULL = C::B_QFULL, B_KFULL = C::B_KFULL, B_KEMPTY = C::B_KEMPTY;
-    constexpr int B_VFULL = C::B_VFULL, B_VEMPTY = C::B_VEMPTY;
+    constexpr int B_VFULL = C::SPLIT_RINGS ? C::B_VFULL : C::B_KFULL, B_VEMPTY = C::B_VEMPTY;
+    constexpr bool SPLIT = C::SPLIT_RINGS;  // without it B_VFULL is B_KFULL and B_KEMPTY is unused
     const PrefillParams& p = tp.base;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -457,15 +462,22 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             // an id outside the pool is out of the tensor's bounds and reads as zeros
             const int coord = used ? id : p.NB;
             const int ks = j % KS, vs = j % VS;
-            if (j >= KS && !wait(B_KEMPTY + ks, ((j / KS) - 1) & 1)) break;
-            if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), TILE_BYTES);
+            if (SPLIT) {
+                if (j >= KS && !wait(B_KEMPTY + ks, ((j / KS) - 1) & 1)) break;
+                if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), TILE_BYTES);
+            } else {
+                if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
+                if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), 2 * TILE_BYTES);
+            }
             __syncwarp();
             if (lane < 4 * NG)
                 tma_load_4d(sbase + OFF_K + ks * TILE_BYTES + tile_off, &kmap, bar(B_KFULL + ks),
                             grp * 64, 0, kvh, coord);
-            if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
-            if (lane == 0) mbar_arrive_expect_tx(bar(B_VFULL + vs), TILE_BYTES);
-            __syncwarp();
+            if (SPLIT) {
+                if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
+                if (lane == 0) mbar_arrive_expect_tx(bar(B_VFULL + vs), TILE_BYTES);
+                __syncwarp();
+            }
             if (lane < 4 * NG)
                 tma_load_4d(sbase + OFF_V + vs * TILE_BYTES + tile_off, &vmap, bar(B_VFULL + vs),
                             grp * 64, 0, kvh, coord);
@@ -501,7 +513,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             const int ks = j % KS, vs = (j + VS - 1) % VS;
             const bool k_next_early =
                 j + 1 < n_steps ? mbar_try_wait(bar(B_KFULL + (j + 1) % KS), ((j + 1) / KS) & 1) : true;
-            const bool v_early = j >= 1 ? mbar_try_wait(bar(B_VFULL + vs), (i / VS) & 1) : true;
+            const bool v_early =
+                SPLIT && j >= 1 ? mbar_try_wait(bar(B_VFULL + vs), (i / VS) & 1) : true;
             const uint64_t k_desc = k_desc0 + (uint64_t)(ks * (TILE_BYTES >> 4));
             const uint64_t v_desc = v_desc0 + (uint64_t)(vs * (TILE_BYTES >> 4));
             const uint32_t s_col = tmem + (j & 1) * STEP, p_col = tmem + ((j + 1) & 1) * STEP;
@@ -520,10 +533,10 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                     }
                     if (leader) tc_commit(bar(tb + T_SFULL + (j & 1)));
                     // the last tile's Q K^T was the last reader of this step's K
-                    if (t == NT - 1 && leader) tc_commit(bar(B_KEMPTY + ks));
+                    if (SPLIT && t == NT - 1 && leader) tc_commit(bar(B_KEMPTY + ks));
                 }
                 if (j >= 1) {  // O[t] += P_{j-1} V_{j-1}
-                    if (t == 0 && !__all_sync(0xffffffffu, v_early)) {
+                    if (SPLIT && t == 0 && !__all_sync(0xffffffffu, v_early)) {
                         ok = wait_all(B_VFULL + vs, (i / VS) & 1);
                         if (!ok) break;
                     }
@@ -545,7 +558,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
                 }
             }
             if (!ok) break;
-            // every tile's P V of the previous step is queued: its V tile may be refilled
+            // every tile's P V of the previous step is queued: its V tile (without split rings,
+            // its K tile too) may be refilled
             if (j >= 1 && leader) tc_commit(bar(B_VEMPTY + vs));
             if (j + 1 < n_steps && !__all_sync(0xffffffffu, k_next_early))
                 ok = wait_all(B_KFULL + (j + 1) % KS, ((j + 1) / KS) & 1);
@@ -951,8 +965,7 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
             (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
         // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
         // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
-        // (head_dim 128; the other head dims scale the tensor work of a step)
-        const double step_us = (nt == 1 ? 0.83 : 0.92) * (D == 256 ? 1.6 : D == 64 ? 0.8 : 1.0);
+        const double step_us = D == 256 ? 1.40 : D == 64 ? (nt == 1 ? 0.66 : 0.88) : (nt == 1 ? 0.83 : 0.92);
         const int64_t s_hi = forced_split_steps ? 1 : std::min<int64_t>({cap_fit, 64, steps_bound / 8});
         for (int64_t s_try = 1; s_try <= std::max<int64_t>(1, s_hi); ++s_try) {
             int64_t T = forced_split_steps ? forced_split_steps : (steps_bound + s_try - 1) / s_try;
