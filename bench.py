@@ -402,8 +402,9 @@ def run_ours(args):
         line["probes"] = bench_probes(torch, api, peak, value / world, achieved)
         line["kv_append"] = bench_append(torch, api, spec, k, v)
         if not args.no_recompute:
+            rshape = tuple(int(x) for x in args.recompute_shape.split(",")) if args.recompute_shape else None
             line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk,
-                                                args.recompute_split)
+                                                args.recompute_split, shape=rshape)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -559,7 +560,7 @@ def bench_append(torch, api, spec, k, v, calls=200):
             "gbps": nbytes / us / 1e3, "bound": "launch latency / host issue rate (2 MB moved per call)"}
 
 
-def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_splits=16):
+def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_splits=16, shape=None):
     """Recomputation recovery of the longest sequence of the batch: causal prefill attention
     over its cached tokens in chunks of `chunk` query tokens (one pa_prefill_split call per
     chunk, context growing, the block table passed no wider than the context).  A dense
@@ -567,6 +568,16 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_spli
     b = int(np.argmax(spec.seq_lens))
     L = int(spec.seq_lens[b])
     H, D = spec.num_q_heads, spec.head_dim
+    if shape is not None:
+        # another layer shape (query heads, KV heads, head_dim): the same sequence length over a
+        # pool of its own with a shuffled block table
+        H, hkv, D = shape
+        nb = (L + 15) // 16
+        k = torch.empty(nb + 64, hkv, 16, D, dtype=torch.bfloat16, device="cuda").normal_()
+        v = torch.empty_like(k).normal_()
+        g = torch.Generator().manual_seed(0x2602)
+        tables = torch.randperm(nb + 64, generator=g)[:nb].to(torch.int32).view(1, nb).cuda()
+        b = 0
     q = torch.empty(L, H, D, dtype=torch.bfloat16, device="cuda").normal_()
     out = torch.empty_like(q)
     tab = tables[b:b + 1].contiguous()
@@ -607,6 +618,7 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_spli
             peak = float(json.load(f)["bf16_tflops"])
     assert int(status.item()) == 0
     return {"tokens": L, "chunk": chunk, "calls": len(calls), "ms": ms, "tflops": flops / ms / 1e9,
+            "shape": {"num_q_heads": H, "num_kv_heads": int(k.shape[1]), "head_dim": D},
             "last_call_launch": {"tiles_per_cta": shapes[-1][0], "kv_split_tokens": shapes[-1][1],
                                  "kv_splits": shapes[-1][2]},
             "bound": "tensor", "peak_tflops": peak,
@@ -859,6 +871,9 @@ def main():
     ap.add_argument("--no-recompute", action="store_true")
     ap.add_argument("--recompute-chunk", type=int, default=512,
                     help="query tokens per pa_prefill call of the recompute leg")
+    ap.add_argument("--recompute-shape", default="",
+                    help="H,Hkv,D of the recompute leg when it should differ from the workload's "
+                         "(e.g. 16,8,256)")
     ap.add_argument("--recompute-split", type=int, default=0,
                     help="kv_split_tokens of the recompute leg (0 = library's choice, -1 = never)")
     ap.add_argument("--cpu-fraction", type=float, default=1.0,

@@ -278,6 +278,15 @@ int pa_prefill_split(const pa_shape* shape, const void* q, const void* k_cache,
                      const int32_t* cu_q_lens, int32_t batch, int32_t total_q, float scale,
                      void* out, void* workspace, size_t workspace_bytes, int32_t kv_split_tokens,
                      int32_t* dev_status, void* cuda_stream);
+/* What pa_prefill_split would launch for these arguments on a GPU with `sm_count` SMs: row
+ * tiles per CTA (0 = the warp-level kernel), split length in tokens (0 = unsplit) and
+ * partial rows per query row.  Host arithmetic only (no GPU is touched): the cost model
+ * behind kv_split_tokens = 0 can be examined, and a caller can size its workspace by trying
+ * sizes.  Returns PA_ERR_WORKSPACE where pa_prefill_split would.  No counterpart in the paper. */
+int pa_prefill_select_launch(const pa_shape* shape, int32_t batch, int32_t total_q,
+                             int32_t max_blocks_per_seq, size_t workspace_bytes,
+                             int32_t kv_split_tokens, int32_t sm_count, int32_t* tiles_per_cta,
+                             int32_t* split_tokens, int32_t* kv_splits);
 /* What the calling thread's last pa_prefill / pa_prefill_split launched: row tiles per CTA (0 =
  * the warp-level kernel), split length in tokens (0 = unsplit) and partial rows per query row.
  * A measurement and test aid; no counterpart in the paper. */

@@ -33,7 +33,7 @@ EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_hos
            "pa_decode_static", "kv_append", "pa_partial_floats", "pa_decode_partial",
            "pa_merge_partials",
            "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_split",
-           "pa_prefill_split_workspace_bytes", "pa_prefill_last_launch", "pa_selftest_wait_expiry", "pa_probe_read"]
+           "pa_prefill_split_workspace_bytes", "pa_prefill_last_launch", "pa_prefill_select_launch", "pa_selftest_wait_expiry", "pa_probe_read"]
 
 
 class PaShape(ctypes.Structure):
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         pi32 = ctypes.POINTER(ctypes.c_int32)
         L.pa_prefill_last_launch.argtypes = [pi32, pi32, pi32]
         L.pa_prefill_last_launch.restype = ctypes.c_int
+        L.pa_prefill_select_launch.argtypes = [pshape, i32, i32, i32, sz, i32, i32, pi32, pi32, pi32]
+        L.pa_prefill_select_launch.restype = ctypes.c_int
         L.pa_selftest_wait_expiry.argtypes = [i32, vp, vp]
         L.pa_selftest_wait_expiry.restype = ctypes.c_int
         L.pa_probe_read.argtypes = [vp, sz, i32, ctypes.c_uint32, vp, vp, vp]
@@ -361,6 +363,17 @@ def pa_prefill_last_launch():
     a, b, c = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
     _check(lib().pa_prefill_last_launch(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
            "pa_prefill_last_launch")
+    return a.value, b.value, c.value
+
+
+def pa_prefill_select_launch(shape: PaShape, batch: int, total_q: int, max_blocks_per_seq: int,
+                             workspace_bytes: int, kv_split_tokens: int = 0, sm_count: int = 148):
+    """Forward to pa_prefill_select_launch (host only): (tiles per CTA, split tokens, splits)."""
+    a, b, c = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(lib().pa_prefill_select_launch(ctypes.byref(shape), batch, total_q, max_blocks_per_seq,
+                                          workspace_bytes, kv_split_tokens, sm_count,
+                                          ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+           "pa_prefill_select_launch")
     return a.value, b.value, c.value
 
 

@@ -44,6 +44,8 @@ __global__ void __launch_bounds__(1024, 1) pa_prefill_plan_kernel(const PrefillP
     __shared__ int s_carry, s_bad;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) s_carry = 0, s_bad = 0;
+    pdl_launch_dependents();
+    pdl_wait();  // the lengths may come from the kernel before; the header is still being read
     __syncthreads();
     for (int base = 0; base < p.batch; base += 1024) {
         const int b = base + tid;
@@ -924,6 +926,7 @@ static size_t prefill_base_bytes(int64_t batch) {
     return (b + 255) & ~(size_t)255;
 }
 
+
 extern "C" int pa_prefill_workspace_bytes(int32_t max_batch, size_t* bytes) {
     if (!bytes) return PA_ERR_NULL;
     if (max_batch < 0) return PA_ERR_ARG;
@@ -944,6 +947,7 @@ extern "C" int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t m
 }
 
 namespace pk {
+
 // Launch shape of the tensor-core path: row tiles per CTA and the KV split length in 64-token
 // steps (0 = no split).  Only bounds are known on the host (the chunk's token count, the
 // longest context the block table can describe), so this is a cost model, not a plan: rounds
@@ -983,7 +987,62 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
     return best;
 }
 static thread_local TcShape g_last_shape = {0, 0, 1};
+
+// What pa_prefill_split launches for these arguments (host arithmetic only).  tiles_per_cta 0
+// = the warp-level kernel.
+static int select_launch(const pa_shape* shape, int batch, int64_t total_q, int max_blocks_per_seq,
+                         size_t workspace_bytes, int kv_split_tokens, int sm_count, TcShape* out) {
+    const int G = shape->num_q_heads / shape->num_kv_heads, H = shape->num_q_heads, D = shape->head_dim;
+    const size_t base_bytes = prefill_base_bytes(batch);
+    if (workspace_bytes < base_bytes) return PA_ERR_WORKSPACE;
+    // tensor-core path: 128-row tiles of (token, head) pairs of one KV-head group
+    static const bool force_mma = [] {
+        const char* e = std::getenv("PAGEDKV_PREFILL");
+        return e && std::string(e) == "mma";
+    }();
+    static const int forced_tiles = [] {
+        const char* e = std::getenv("PAGEDKV_PREFILL_TILES");
+        const int v = e ? std::atoi(e) : 0;
+        return v == 1 || v == 2 ? v : 0;
+    }();
+    *out = TcShape{0, 0, 1};
+    if (force_mma) return PA_OK;
+    const int64_t steps_bound = std::max<int64_t>(1, ((int64_t)max_blocks_per_seq * BS + 63) / 64);
+    const size_t per_split = (size_t)std::max<int64_t>(total_q, 1) * H * (D + 2) * sizeof(float);
+    const int64_t cap_fit = (int64_t)((workspace_bytes - base_bytes) / per_split);
+    int forced_steps = 0;
+    if (kv_split_tokens > 0) {
+        forced_steps = (kv_split_tokens + 63) / 64;
+        if (forced_steps >= steps_bound) kv_split_tokens = -1;  // one split covers everything
+        else if ((steps_bound + forced_steps - 1) / forced_steps > cap_fit) return PA_ERR_WORKSPACE;
+    }
+    *out = kv_split_tokens < 0
+               ? choose_tc_shape(total_q, batch, shape->num_kv_heads, G, H, D, steps_bound, sm_count,
+                                 1, forced_tiles, 0)
+               : choose_tc_shape(total_q, batch, shape->num_kv_heads, G, H, D, steps_bound, sm_count,
+                                 cap_fit, forced_tiles, forced_steps);
+    return PA_OK;
+}
 }  // namespace pk
+
+extern "C" int pa_prefill_select_launch(const pa_shape* shape, int32_t batch, int32_t total_q,
+                                        int32_t max_blocks_per_seq, size_t workspace_bytes,
+                                        int32_t kv_split_tokens, int32_t sm_count,
+                                        int32_t* tiles_per_cta, int32_t* split_tokens,
+                                        int32_t* kv_splits) {
+    if (!shape || !tiles_per_cta || !split_tokens || !kv_splits) return PA_ERR_NULL;
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (batch <= 0 || total_q <= 0 || max_blocks_per_seq < 0 || sm_count <= 0) return PA_ERR_ARG;
+    TcShape ts;
+    rc = select_launch(shape, batch, total_q, max_blocks_per_seq, workspace_bytes, kv_split_tokens,
+                       sm_count, &ts);
+    if (rc) return rc;
+    *tiles_per_cta = ts.tiles_per_cta;
+    *split_tokens = ts.split_steps * 64;
+    *kv_splits = ts.split_cap;
+    return PA_OK;
+}
 
 extern "C" int pa_prefill_last_launch(int32_t* tiles_per_cta, int32_t* kv_split_tokens,
                                       int32_t* kv_splits) {
@@ -1033,45 +1092,33 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
     plan.batch = batch;
     plan.max_blocks = max_blocks_per_seq;
     plan.total_q = total_q;
-    // tensor-core path: 128-row tiles of (token, head) pairs of one KV-head group
-    static const bool force_mma = [] {
-        const char* e = std::getenv("PAGEDKV_PREFILL");
-        return e && std::string(e) == "mma";
-    }();
-    const bool use_tc = !force_mma && (D == 64 || D == 128 || D == 256) && G <= 128;
-    static const int forced_tiles = [] {
-        const char* e = std::getenv("PAGEDKV_PREFILL_TILES");
-        const int v = e ? std::atoi(e) : 0;
-        return v == 1 || v == 2 ? v : 0;
-    }();
-    TcShape ts = {1, 0, 1};
-    if (use_tc) {
-        const int64_t steps_bound = std::max<int64_t>(1, ((int64_t)max_blocks_per_seq * BS + 63) / 64);
-        const size_t per_split = (size_t)total_q * H * (D + 2) * sizeof(float);
-        const int64_t cap_fit = (int64_t)((workspace_bytes - base_bytes) / per_split);
-        int forced_steps = 0;
-        if (kv_split_tokens > 0) {
-            forced_steps = (kv_split_tokens + 63) / 64;
-            if (forced_steps >= steps_bound) kv_split_tokens = -1;  // one split covers everything
-            else if ((steps_bound + forced_steps - 1) / forced_steps > cap_fit) return PA_ERR_WORKSPACE;
-        }
-        if (kv_split_tokens < 0)
-            ts = choose_tc_shape(total_q, batch, shape->num_kv_heads, G, H, D, steps_bound,
-                                 dev.sm_count, 1, forced_tiles, 0);
-        else
-            ts = choose_tc_shape(total_q, batch, shape->num_kv_heads, G, H, D, steps_bound,
-                                 dev.sm_count, cap_fit, forced_tiles, forced_steps);
-    }
+    TcShape ts = {0, 0, 1};
+    rc = select_launch(shape, batch, total_q, max_blocks_per_seq, workspace_bytes, kv_split_tokens,
+                       dev.sm_count, &ts);
+    if (rc) return rc;
+    const bool use_tc = ts.tiles_per_cta != 0;
     g_last_shape = use_tc ? ts : TcShape{0, 0, 1};
     plan.tpg = use_tc ? ts.tiles_per_cta * (128 / G) : 16 / G;  // 128 / G rounds down
     plan.split_steps = ts.split_steps;
     plan.hdr = hdr;
     plan.gstart = hdr + PF_WORDS;
     plan.status = dev_status ? dev_status : hdr + PF_STATUS;
-    pa_prefill_plan_kernel<<<1, 1024, 0, st>>>(plan);
-    count_launch();
-    rc = check_cuda(cudaGetLastError());
-    if (rc) return rc;
+    {
+        // launched as a programmatic dependent of whatever precedes it in the stream (the
+        // previous chunk's merge): its launch latency hides under that kernel's tail
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1);
+        cfg.blockDim = dim3(1024);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        count_launch();
+        rc = check_cuda(cudaLaunchKernelEx(&cfg, pa_prefill_plan_kernel, plan));
+        if (rc) return rc;
+    }
 
     PrefillParams pp;
     pp.q = static_cast<const __nv_bfloat16*>(q);
