@@ -168,12 +168,23 @@ def sample_kv_bytes(spec, lens):
 # --------------------------------------------------------------------------------------
 # swap timing (N = 1 only)
 # --------------------------------------------------------------------------------------
+def make_pools(torch, wl, layers, nb, hkv, d, layout, seed_k, seed_v, dev):
+    """K and V pools as [layers, NB, Hkv, 16, D] views.  "layer": each layer's blocks together
+    (one layer's attention stays inside NB x 32 KiB); "block": all layers of a block together
+    (a block's whole payload is one contiguous piece, ideal for swapping, while one layer's
+    attention then touches every page of the pool)."""
+    n = nb * hkv * 16 * d
+    if layout == "layer":
+        return (wl.normal_bf16_torch(0, layers * n, seed_k, dev).view(layers, nb, hkv, 16, d),
+                wl.normal_bf16_torch(0, layers * n, seed_v, dev).view(layers, nb, hkv, 16, d))
+    store = wl.normal_bf16_torch(0, 2 * layers * n, seed_k, dev).view(nb, layers, 2, hkv, 16, d)
+    return store[:, :, 0].permute(1, 0, 2, 3, 4), store[:, :, 1].permute(1, 0, 2, 3, 4)
+
+
 def bench_swap(args, torch, api, wl, decode_step, decode_bytes):
     dev = "cuda"
     layers, hkv, d, nb = 32, 8, 128, args.swap_pool_blocks
-    n_elems = layers * nb * hkv * 16 * d
-    k_pool = wl.normal_bf16_torch(0, n_elems, 0x51, dev).view(layers, nb, hkv, 16, d)
-    v_pool = wl.normal_bf16_torch(0, n_elems, 0x52, dev).view(layers, nb, hkv, 16, d)
+    k_pool, v_pool = make_pools(torch, wl, layers, nb, hkv, d, args.pool_layout, 0x51, 0x52, dev)
     bb = api.kv_block_bytes(k_pool, v_pool)
     tokens = [int(t) for t in args.swap_tokens.split(",")]
     max_blocks = max(tokens) // 16
@@ -219,6 +230,31 @@ def bench_swap(args, torch, api, wl, decode_step, decode_bytes):
                          "in_frac_of_link": nbytes / t_in / 1e6 / link["h2d_gbps"]}
         rows.append(row)
 
+    # reference point: no kernel at all, one cudaMemcpyAsync per contiguous piece of the
+    # smallest eviction (32 KiB per (block, layer, K|V) in the layer layout, a block's whole
+    # 2 MiB in the block layout), issued from this Python loop
+    n = tokens[0] // 16
+    src = rng.permutation(nb)[:n]
+    img = host[:n * bb].view(torch.bfloat16).view(n, layers, 2, hkv, 16, d)
+
+    def naive_out():
+        for i, b in enumerate(src.tolist()):
+            if args.pool_layout == "block":   # K and V of all layers of block b are adjacent
+                blk = hkv * 16 * d
+                img[i].copy_(k_pool[:, b].as_strided((layers, 2, hkv, 16, d),
+                                                     (2 * blk, blk, 16 * d, d, 1)),
+                             non_blocking=True)
+            else:
+                for l in range(layers):
+                    img[i, l, 0].copy_(k_pool[l, b], non_blocking=True)
+                    img[i, l, 1].copy_(v_pool[l, b], non_blocking=True)
+
+    t_naive = timed(naive_out, reps=2)
+    naive = {"tokens": tokens[0], "bytes": n * bb,
+             "copies": n * (1 if args.pool_layout == "block" else 2 * layers),
+             "out_gbps": n * bb / t_naive / 1e6,
+             "out_frac_of_link": n * bb / t_naive / 1e6 / link["d2h_gbps"]}
+
     # churn: evict + restore on the side stream while decode steps run on the main stream
     n = tokens[-1] // 16
     perm = rng.permutation(nb)
@@ -255,8 +291,9 @@ def bench_swap(args, torch, api, wl, decode_step, decode_bytes):
              "decode_overlapped_gbps": steps * decode_bytes / e[2].elapsed_time(e[3]) / 1e6,
              "decode_steps_during_swap": steps}
     return {"pool": {"layers": layers, "kv_heads": hkv, "head_dim": d, "blocks": nb,
-                     "block_bytes": bb, "staging_mib": args.swap_staging_mib},
-            "host_link": link, "sizes": rows, "churn": churn}
+                     "block_bytes": bb, "staging_mib": args.swap_staging_mib,
+                     "layout": args.pool_layout},
+            "host_link": link, "sizes": rows, "memcpy_per_piece": naive, "churn": churn}
 
 
 # --------------------------------------------------------------------------------------
@@ -331,6 +368,33 @@ def run_ours(args):
     torch.cuda.synchronize()
     api.pa_profile_enable(False)
     plan_ms, attn_ms, comb_ms, calls = api.pa_profile_read()
+    # third region: the step captured once into a CUDA graph and replayed K times (the launch
+    # cost of the three kernels leaves the host; reported beside `value`, never instead of it)
+    graph_ms = graph_err = None
+    if world == 1:
+        try:
+            cap = torch.cuda.Stream()
+            cap.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(cap):
+                step()                                  # set-up calls happen outside the capture
+                cap.synchronize()
+                with torch.cuda.graph(g, stream=cap):
+                    api.pa_decode(q, k, v, tables, lens, spec.scale, out, ws, dev_status=status,
+                                  partition_tokens=args.partition_tokens, stream=cap)
+                for _ in range(3):
+                    g.replay()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(cap)
+                for _ in range(args.steps):
+                    g.replay()
+                g1.record(cap)
+                g1.synchronize()
+                graph_ms = g0.elapsed_time(g1) / args.steps
+            stream.wait_stream(cap)
+        except Exception as exc:  # a capture that the driver refuses is reported, not fatal
+            graph_err = str(exc)[:200]
+            torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     ms, total_bytes = aggregate_over_ranks(ms_local, float(step_bytes) * args.steps, dist)
@@ -390,6 +454,9 @@ def run_ours(args):
         "e2e": {"value": bytes_e2e / ms_e2e / 1e6, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
+        "graph_replay": {"ms_per_step": graph_ms,
+                         "value": (step_bytes / graph_ms / 1e6) if graph_ms else None,
+                         "error": graph_err},
         "kernels_ms_per_step": {"plan": plan_ms / max(calls, 1), "attention": attn_avg_ms,
                                 "combine": comb_ms / max(calls, 1)},
         "roofline": {"bound": "hbm", "kernel": "pa_decode_kernel", "achieved": achieved,
@@ -745,9 +812,8 @@ def run_churn(args):
     spec = wl.config_spec(4)
     layers, nb = spec.num_layers, spec.num_blocks
     n = nb * spec.block_elems
-    shape5 = (layers, nb, spec.num_kv_heads, 16, spec.head_dim)
-    k_pool = wl.normal_bf16_torch(0, layers * n, spec.seed_k, dev).view(shape5)
-    v_pool = wl.normal_bf16_torch(0, layers * n, spec.seed_v, dev).view(shape5)
+    k_pool, v_pool = make_pools(torch, wl, layers, nb, spec.num_kv_heads, spec.head_dim,
+                                args.pool_layout, spec.seed_k, spec.seed_v, dev)
     q = wl.q_torch(spec, dev)
     tables = torch.from_numpy(spec.block_tables).to(dev)
     out = torch.empty_like(q)
@@ -847,7 +913,7 @@ def run_churn(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": spec.name, "batch": spec.batch, "layers": layers,
                    "pool_blocks": nb, "allocated_blocks": nb - len(spec.free_blocks),
-                   "pool_bytes": 2 * layers * n * 2, "block_bytes": bb,
+                   "pool_bytes": 2 * layers * n * 2, "block_bytes": bb, "pool_layout": args.pool_layout,
                    "total_context_tokens": spec.total_tokens,
                    "step": "32 pa_decode calls (one per layer, plan reused) over the non-evicted batch",
                    "staging_mib": args.swap_staging_mib},
@@ -890,6 +956,9 @@ def main():
     ap.add_argument("--cpu-fraction", type=float, default=1.0,
                     help="fraction of the batch's tokens the CPU baseline pass covers")
     ap.add_argument("--swap-pool-blocks", type=int, default=6144)
+    ap.add_argument("--pool-layout", default="layer", choices=["layer", "block"],
+                    help="multi-layer pools of the swap legs and of workload 4: each layer's blocks "
+                         "together, or all layers of a block together")
     ap.add_argument("--swap-tokens", default="1024,4096,16384")
     ap.add_argument("--swap-staging-mib", type=int, default=256)
     args = ap.parse_args()
