@@ -102,3 +102,53 @@ def test_cfg1_eviction_round_trip_keeps_decode_bits():
     g.tables.copy_(torch.from_numpy(t))
     after = g.run()
     assert torch.equal(after.view(torch.int16), before.view(torch.int16))
+
+
+@pytest.mark.parametrize("staged", [False, True])
+def test_block_major_pool_swap_and_per_layer_decode(staged):
+    # all layers of a block stored together ([NB][layer][K|V][Hkv][16][D]): the pools handed to
+    # the library are strided views; swaps stay bit-exact, every other byte (the other blocks
+    # of the interleaved store) stays untouched, and decode on one layer's view matches the
+    # oracle with a block stride of layers * 2 * 32 KiB
+    layers, NB, Hkv, D, H = 3, 48, 2, 128, 8
+    k, v = make_pools(layers, NB, Hkv, D, seed=77)
+    store = torch.empty(NB, layers, 2, Hkv, 16, D, dtype=torch.bfloat16, device="cuda")
+    store[:, :, 0] = bits_to_torch(k).permute(1, 0, 2, 3, 4)
+    store[:, :, 1] = bits_to_torch(v).permute(1, 0, 2, 3, 4)
+    kd, vd = store[:, :, 0].permute(1, 0, 2, 3, 4), store[:, :, 1].permute(1, 0, 2, 3, 4)
+    assert kd.stride(1) == layers * 2 * Hkv * 16 * D and not kd.is_contiguous()
+    rng = np.random.default_rng(7)
+    perm = rng.permutation(NB)
+    src, dst = perm[:9].astype(np.int32), perm[9:18].astype(np.int32)
+    bb = api.kv_block_bytes(kd, vd)
+    host = torch.zeros(9 * bb, dtype=torch.uint8).pin_memory()
+    staging = torch.empty(4 * bb, dtype=torch.uint8, device="cuda") if staged else None
+    api.kv_swap_out(kd, vd, src, host, staging)
+    torch.cuda.synchronize()
+    image = oracle.swap_out(k, v, src)
+    assert (host.numpy().view(np.uint16) == image.reshape(-1)).all()
+    # in this layout a block's image is the block's own bytes
+    assert (as_bits(store[int(src[0])]).reshape(-1) == image.reshape(9, -1)[0]).all()
+    api.kv_swap_in(kd, vd, host, dst, staging)
+    torch.cuda.synchronize()
+    k2, v2 = k.copy(), v.copy()
+    oracle.swap_in(k2, v2, image, dst)
+    assert (as_bits(kd) == k2).all() and (as_bits(vd) == v2).all()
+    # decode over layer 1 of the restored pool, tables pointing at the new ids
+    lens = np.array([9 * 16 - 5, 40], np.int32)
+    tables = np.full((2, 9), -1, np.int32)
+    tables[0] = dst
+    tables[1, :3] = perm[20:23]
+    q = wl.normal_bf16_np(0, 2 * H * D, 78).reshape(2, H, D)
+    qd = bits_to_torch(q)
+    out = torch.empty_like(qd)
+    shape = api.shape_of(kd[1], H)
+    ws = torch.empty(api.pa_workspace_bytes(shape, 2, 16 * tables.size), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.pa_decode(qd, kd[1], vd[1], torch.from_numpy(tables).cuda(), torch.from_numpy(lens).cuda(),
+                  D ** -0.5, out, ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = oracle.pa_decode(q, k2[1], v2[1], tables, lens, np.float32(D ** -0.5))
+    from helpers import assert_parity, torch_to_f64
+    assert_parity(torch_to_f64(out), ref, "block-major layer view")
