@@ -1071,6 +1071,7 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
         return PA_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return PA_ERR_ALIGN;
     if ((int64_t)max_blocks_per_seq * BS > INT32_MAX) return PA_ERR_ARG;
+    if ((int64_t)total_q * shape->num_q_heads / 8 >= INT32_MAX) return PA_ERR_ARG;  // rows of the merge grid
     const size_t base_bytes = prefill_base_bytes(batch);
     if (workspace_bytes < base_bytes) return PA_ERR_WORKSPACE;
     DeviceInfo dev;
