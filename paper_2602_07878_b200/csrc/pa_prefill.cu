@@ -1,8 +1,12 @@
 // Chunked causal prefill over the paged KV cache (the recomputation path of a preempted
 // sequence): every query token of the chunk attends to the cached tokens up to its own
-// position.  First implementation: the same independent-warp machinery as decode -- a warp
-// owns 16 query rows (tokens x heads of one KV-head group) and streams the KV blocks they may
-// see through its private TMA ring; neighbouring warps re-read the same blocks from L2.
+// position.  Two implementations behind pa_prefill / pa_prefill_split:
+//   * pa_prefill_tc_kernel: tcgen05 tensor cores, 128-row tiles, scores, weights and output
+//     accumulator in tensor memory, optionally the KV range of a tile split over CTAs with
+//     pa_prefill_merge_kernel combining the partial rows (every supported shape);
+//   * pa_prefill_kernel: the independent-warp machinery of decode -- a warp owns 16 query rows
+//     (tokens x heads of one KV-head group) and streams the KV blocks they may see through
+//     its private TMA ring; selected with PAGEDKV_PREFILL=mma, kept as a second implementation.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -272,16 +276,16 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 
 
 // ======================================================================================
-// tcgen05 version: one CTA = 128 query rows ((token, head) pairs of one KV-head group)
+// tcgen05 version: a row tile = 128 query rows ((token, head) pairs of one KV-head group)
 // ======================================================================================
-// Warps 0-3: softmax and epilogue (thread i owns row i = TMEM lane i); warp 4: TMA producer;
-// warp 5: MMA issuer.  Per 64-token KV step:  S = Q K^T (M 128, N 64, K 128) into one of two
-// TMEM score buffers, the softmax warps turn S into bf16 weights P written back over the
-// first 32 columns of that score buffer (and rescale the TMEM accumulator O when a row
-// maximum has grown by more than 2^8), then O += P V (M 128, N 128, K 64) with P read from
-// tensor memory: the weights never touch shared memory, whose bandwidth the two MMAs'
-// operand reads already fill.  Two score buffers and four KV stages let Q K^T of step j+1
-// overlap the softmax of step j.
+// Warps 0 .. 4 NT - 1: softmax and epilogue, four per tile (thread i of a tile's warps owns
+// row i = TMEM lane i); then one TMA producer warp and one MMA warp.  Per 64-token KV step and
+// tile: S = Q K^T (M 128, N 64, K head_dim) into one of two TMEM score buffers, the softmax
+// warps turn S into bf16 weights P written back over the first 32 columns of that score
+// buffer (and rescale the TMEM accumulator O when a row maximum has grown by more than 2^8),
+// then O += P V (M 128, N head_dim, K 64) with P read from tensor memory: the weights never
+// touch shared memory, whose bandwidth the MMAs' operand reads already fill.  Two score
+// buffers and a ring of K/V tiles let Q K^T of step j+1 overlap the softmax of step j.
 namespace tc {
 constexpr int ROWS = 128, STEP = 64;
 #ifndef PAGEDKV_POLY_PAIRS
