@@ -194,3 +194,51 @@ def test_decode_time_is_linear_in_total_context_once_bandwidth_bound():
         del k, v
     assert 1.8 < times[2] / times[1] < 2.2, times
     assert 1.8 < times[4] / times[2] < 2.2, times
+
+
+@pytest.mark.parametrize("H,Hkv,D,chunk", [(32, 8, 128, 512), (32, 8, 128, 32768), (16, 8, 256, 512),
+                                           (16, 8, 256, 8192)])
+def test_full_size_recompute_sampled_against_oracle(H, Hkv, D, chunk):
+    """The recompute leg of bench.py at its sizes: the last `chunk` query tokens of a
+    32768-token context over a shuffled block table, launched as the bench launches it
+    (library-chosen tile count and KV split, workspace for 16 splits).  The oracle recomputes
+    sampled query tokens one by one -- a query at position p is a decode step over p + 1 tokens
+    -- on the first and last rows of the chunk, around tile and split boundaries and at random."""
+    L, dev = 32768, "cuda"
+    nb = L // 16
+    kb = wl.normal_bf16_np(0, (nb + 64) * Hkv * 16 * D, 901).reshape(nb + 64, Hkv, 16, D)
+    vb = wl.normal_bf16_np(0, (nb + 64) * Hkv * 16 * D, 902).reshape(nb + 64, Hkv, 16, D)
+    table = np.random.default_rng(903).permutation(nb + 64)[:nb].astype(np.int32).reshape(1, nb)
+    qb = wl.normal_bf16_np(0, chunk * H * D, 904).reshape(chunk, H, D)
+    from helpers import bits_to_torch
+    k, v, q = bits_to_torch(kb), bits_to_torch(vb), bits_to_torch(qb)
+    out = torch.full_like(q, float("nan"))
+    ws = torch.empty(api.pa_prefill_split_workspace_bytes(api.shape_of(k, H), 1, chunk, 16),
+                     dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    api.pa_prefill_split(q, k, v, torch.from_numpy(table).to(dev),
+                         torch.tensor([L], dtype=torch.int32, device=dev),
+                         torch.tensor([0, chunk], dtype=torch.int32, device=dev), D ** -0.5, out, ws,
+                         dev_status=status)
+    torch.cuda.synchronize()
+    tiles, split_tok, splits = api.pa_prefill_last_launch()
+    assert int(status.item()) == 0 and tiles in (1, 2)
+    if chunk == 512:
+        assert splits >= 2                       # few tiles, long context: the KV range is split
+    assert torch.isfinite(out).all()
+    # rows are convex mixtures of table values
+    assert float(out.float().abs().max()) <= float(v.float().abs().max())
+    rng = np.random.default_rng(905)
+    tpt = 128 // (H // Hkv)
+    picks = {0, 1, chunk - 1, chunk - 2, tpt - 1, tpt, 2 * tpt - 1, 2 * tpt, chunk // 2}
+    if split_tok:                                # queries whose position sits at a split boundary
+        first = L - chunk
+        for s in range(1, splits):
+            t = s * split_tok - first
+            picks |= {x for x in (t - 1, t, t + 1) if 0 <= x < chunk}
+    picks |= {int(x) for x in rng.integers(0, chunk, 8)}
+    toks = sorted(picks)
+    pos = np.array([L - chunk + t for t in toks], np.int32)
+    ref = oracle.pa_decode(qb[toks], kb, vb, np.repeat(table, len(toks), axis=0), pos + 1,
+                           np.float32(D ** -0.5))
+    assert_parity(torch_to_f64(out[toks]), ref, f"recompute H{H}/{Hkv} D{D} chunk {chunk}")
