@@ -471,7 +471,8 @@ def run_ours(args):
         if not args.no_recompute:
             rshape = tuple(int(x) for x in args.recompute_shape.split(",")) if args.recompute_shape else None
             line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk,
-                                                args.recompute_split, shape=rshape)
+                                                args.recompute_split, shape=rshape,
+                                                cpu=not args.no_cpu)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -627,7 +628,8 @@ def bench_append(torch, api, spec, k, v, calls=200):
             "gbps": nbytes / us / 1e3, "bound": "launch latency / host issue rate (2 MB moved per call)"}
 
 
-def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_splits=16, shape=None):
+def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_splits=16, shape=None,
+                    cpu=False):
     """Recomputation recovery of the longest sequence of the batch: causal prefill attention
     over its cached tokens in chunks of `chunk` query tokens (one pa_prefill_split call per
     chunk, context growing, the block table passed no wider than the context).  A dense
@@ -691,7 +693,30 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_spli
             peak = float(peaks["bf16_tflops"])
             sustained = float(peaks.get("bf16_tflops_sustained", 0.0)) or None
     assert int(status.item()) == 0
+    cpu_part = None
+    if cpu:
+        # the prefill oracle, as it stands, on the last 16 query tokens of the sequence (the
+        # sequence's blocks copied to the host in table order), timed and compared with the
+        # rows the last call wrote
+        import oracle
+
+        n_s = min(16, L)
+        nb_seq = (L + 15) // 16
+        ids = tab[0, :nb_seq].long()
+        to_bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+        kh, vh, qh = to_bits(k[ids]), to_bits(v[ids]), to_bits(q[L - n_s:])
+        t0 = time.perf_counter()
+        ref = oracle.pa_prefill(qh, kh, vh, np.arange(nb_seq, dtype=np.int32)[None], [L], [0, n_s],
+                                spec.scale)
+        dt = time.perf_counter() - t0
+        got = out[L - n_s:].float().cpu().numpy().astype(np.float64)
+        err = np.abs(got - ref).max(axis=-1) / np.abs(ref).max(axis=-1)
+        cpu_part = {"value": 4.0 * D * H * n_s * (2 * L - n_s + 1) / 2 / dt / 1e12, "unit": "TFLOP/s",
+                    "cores": oracle.threads(), "kind": "oracle", "seconds": dt,
+                    "sample": f"the last {n_s} of {L} query tokens, one pass",
+                    "max_row_rel_err_of_gpu_rows": float(err.max())}
     return {"tokens": L, "chunk": chunk, "calls": len(calls), "ms": ms, "tflops": flops / ms / 1e9,
+            "cpu_baseline": cpu_part,
             "shape": {"num_q_heads": H, "num_kv_heads": int(k.shape[1]), "head_dim": D},
             "clocks": cs.summary(),
             "last_call_launch": {"tiles_per_cta": shapes[-1][0], "kv_split_tokens": shapes[-1][1],
