@@ -472,7 +472,7 @@ def run_ours(args):
             rshape = tuple(int(x) for x in args.recompute_shape.split(",")) if args.recompute_shape else None
             line["recompute"] = bench_recompute(torch, api, spec, k, v, tables, args.recompute_chunk,
                                                 args.recompute_split, shape=rshape,
-                                                cpu=not args.no_cpu)
+                                                cpu=not args.no_cpu, clock_ms=args.recompute_clock_ms)
         if not args.no_swap:
             line["swap"] = bench_swap(args, torch, api, wl, step, step_bytes)
         if not args.no_cpu:
@@ -629,7 +629,7 @@ def bench_append(torch, api, spec, k, v, calls=200):
 
 
 def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_splits=16, shape=None,
-                    cpu=False):
+                    cpu=False, clock_ms=500.0):
     """Recomputation recovery of the longest sequence of the batch: causal prefill attention
     over its cached tokens in chunks of `chunk` query tokens (one pa_prefill_split call per
     chunk, context growing, the block table passed no wider than the context).  A dense
@@ -679,7 +679,7 @@ def bench_recompute(torch, api, spec, k, v, tables, chunk=512, split=0, max_spli
     ms = e0.elapsed_time(e1)
     # clocks under this load: the leg repeated for about half a second while NVML is sampled
     with ClockSampler(torch.cuda.current_device()) as cs:
-        for _ in range(max(1, int(500.0 / max(ms, 1e-3)))):
+        for _ in range(int(clock_ms / max(ms, 1e-3))):
             run()
         torch.cuda.synchronize()
     # 4 * D flops per (query, visible key, head): QK^T and PV, 2 flops per multiply-add
@@ -976,6 +976,9 @@ def main():
     ap.add_argument("--recompute-shape", default="",
                     help="H,Hkv,D of the recompute leg when it should differ from the workload's "
                          "(e.g. 16,8,256)")
+    ap.add_argument("--recompute-clock-ms", type=float, default=500.0,
+                    help="how long the recompute leg is repeated while the clocks are sampled "
+                         "(0 = not at all, e.g. under a profiler)")
     ap.add_argument("--recompute-split", type=int, default=0,
                     help="kv_split_tokens of the recompute leg (0 = library's choice, -1 = never)")
     ap.add_argument("--cpu-fraction", type=float, default=1.0,
