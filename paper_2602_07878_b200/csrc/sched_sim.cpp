@@ -253,11 +253,13 @@ extern "C" int sched_step(void* sched, sched_step_out* out) {
         bool self_evicted = false;
         while (S.free_blocks.empty()) {
             const int victim = pick_victim(S);
+            const size_t vpos = std::find(S.running.begin(), S.running.end(), victim) - S.running.begin();
             preempt(S, victim);
             if (victim == idx) {
                 self_evicted = true;
                 break;
             }
+            if (vpos < i) --i;  // a victim ahead of this sequence left the list: positions shift
         }
         if (self_evicted) continue;  // running shrank; position i now holds the next sequence
         S.take(s, 1);

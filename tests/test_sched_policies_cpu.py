@@ -139,3 +139,47 @@ def test_fairness_switches_shorten_the_short_requests_wait_under_a_squeeze():
     assert quota_ttft < base_ttft and quota_steps < base_steps
     # every request still finishes under the fairness switches (no starvation in this mix)
     assert fair_steps < 4 * base_steps
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_traffic_under_random_policies_keeps_the_invariants(seed):
+    """Whatever the switches: no physical block is ever in two tables of one iteration, the
+    token budget holds, swapped blocks come back, everything drains and every block returns to
+    the free list; quotas bound what a request generates and holds."""
+    rng = np.random.default_rng(1000 + seed)
+    policy = dict(victim_policy=int(rng.integers(0, 2)), demote_victims=bool(rng.integers(0, 2)),
+                  admit_lookahead=int(rng.integers(0, 6)),
+                  max_output_tokens=int(rng.choice([0, 40, 150])),
+                  max_seq_blocks=int(rng.choice([0, 12, 30])))
+    mode = int(rng.integers(0, 2))
+    s = Scheduler(num_blocks=160, max_num_seqs=24, max_batched_tokens=192, max_blocks_per_seq=48,
+                  host_blocks=int(rng.choice([0, 40, 400])), preempt_mode=mode)
+    s.set_policy(**policy)
+    n_req, added = 90, 0
+    for step in range(200000):
+        while added < n_req and added <= step // 2:           # arrivals spread over time
+            assert s.add_request(added, int(rng.integers(1, 300)), int(rng.integers(1, 260)))
+            added += 1
+        st = s.step()
+        if st.idle and added == n_req:
+            break
+        used = set()
+        for tab, lens in ((st.decode_tables, st.decode_lens), (st.prefill_tables, st.prefill_ctx_lens)):
+            for row, L in zip(tab, lens):
+                blk = [int(b) for b in row[: (int(L) + 15) // 16]]
+                assert all(0 <= b < 160 for b in blk) and not (used & set(blk)), policy
+                if policy["max_seq_blocks"]:
+                    assert len(blk) <= max(policy["max_seq_blocks"], 1 + 299 // 16), policy
+                used |= set(blk)
+        assert int(st.prefill_q_lens.sum()) + len(st.decode_ids) <= 192
+        assert not (set(int(b) for b in st.swap_in_blocks) - used)   # restored blocks are in use
+    else:
+        raise AssertionError(f"did not drain under {policy}")
+    stt = s.stats()
+    assert stt.finished == n_req and stt.free_blocks == 160 and stt.running == 0 and stt.waiting == 0
+    assert stt.swapped_in_blocks == stt.swapped_out_blocks
+    for i in range(n_req):
+        r = s.request_stats(i)
+        assert r.finished_step >= r.first_token_step >= r.queued_step >= 0 or r.generated == 0
+        if policy["max_output_tokens"]:
+            assert r.generated <= policy["max_output_tokens"]
