@@ -8,7 +8,11 @@ from paper_2602_07878_b200 import api
 from paper_2602_07878_b200 import workloads as wl
 
 # Tolerance for bf16 inputs with fp32 accumulation: element-wise |gpu - ref| <= 1e-2 and,
-# per (sequence, head) row, max_d |gpu - ref| <= 2e-2 * max_d |ref|.
+# per (sequence, head) row, max_d |gpu - ref| <= 2e-2 * max_d |ref|.  The output is bf16:
+# from 2 upwards its values are 2^-6 apart (2^-5 from 4), so rounding the result alone takes
+# up to 7.8e-3 (1.6e-2) and the bf16 rounding of the softmax weights adds up to 2^-9 of the
+# magnitude; there the element-wise bound is one spacing of bf16 at |ref| instead of 1e-2.
+# Outputs that large need a softmax that is nearly one-hot on an extreme element of V.
 ABS_TOL = 1e-2
 REL_TOL = 2e-2
 GUARD = 4096            # guard elements on each side of a test's output buffer
@@ -20,7 +24,9 @@ def assert_parity(gpu: np.ndarray, ref: np.ndarray, what: str = "", abs_tol: flo
     assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
     assert np.isfinite(gpu).all(), f"{what}: non-finite output"
     err = np.abs(gpu - ref)
-    assert err.max(initial=0.0) <= abs_tol, f"{what}: abs err {err.max():.3e}"
+    spacing = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7)   # of bf16 at |ref|
+    excess = err - np.maximum(abs_tol, np.where(np.abs(ref) >= 2.0, spacing, 0.0))
+    assert excess.max(initial=-1.0) <= 0.0, f"{what}: abs err {err.max():.3e}"
     row_err = err.reshape(-1, err.shape[-1]).max(axis=1)
     row_ref = np.abs(ref).reshape(-1, ref.shape[-1]).max(axis=1)
     rel = row_err / np.maximum(row_ref, 1e-30)
