@@ -80,3 +80,48 @@ def test_random_prefill_cases(seed):
     ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
     assert_parity(torch_to_f64(out), ref,
                   f"prefill seed {seed}: H{H}/{Hkv} D{D} split {split} ctx {ctx} q {qlens}")
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_swap_and_append_cases_are_bit_exact(seed):
+    rng = np.random.default_rng(9000 + seed)
+    layers, Hkv, D = int(rng.integers(1, 6)), int(rng.choice([1, 2, 8])), int(rng.choice([64, 128, 256]))
+    NB = int(rng.integers(8, 120))
+    n = layers * NB * Hkv * 16 * D
+    k = wl.normal_bf16_np(0, n, 9100 + seed).reshape(layers, NB, Hkv, 16, D)
+    v = wl.normal_bf16_np(0, n, 9200 + seed).reshape(layers, NB, Hkv, 16, D)
+    kd, vd = bits_to_torch(k), bits_to_torch(v)
+    if rng.integers(0, 2):   # all layers of a block stored together
+        store = torch.empty(NB, layers, 2, Hkv, 16, D, dtype=torch.bfloat16, device="cuda")
+        store[:, :, 0], store[:, :, 1] = kd.permute(1, 0, 2, 3, 4), vd.permute(1, 0, 2, 3, 4)
+        kd, vd = store[:, :, 0].permute(1, 0, 2, 3, 4), store[:, :, 1].permute(1, 0, 2, 3, 4)
+    as_bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    m = int(rng.integers(1, NB // 2 + 1))
+    perm = rng.permutation(NB)
+    src, dst = perm[:m].astype(np.int32), perm[m:2 * m].astype(np.int32)
+    bb = api.kv_block_bytes(kd, vd)
+    host = torch.zeros(m * bb, dtype=torch.uint8).pin_memory()
+    staging = (torch.empty(int(rng.integers(1, m + 1)) * bb, dtype=torch.uint8, device="cuda")
+               if rng.integers(0, 2) else None)
+    api.kv_swap_out(kd, vd, src, host, staging)
+    torch.cuda.synchronize()
+    image = oracle.swap_out(k, v, src)
+    assert (host.numpy().view(np.uint16) == image.reshape(-1)).all()
+    api.kv_swap_in(kd, vd, host, dst, staging)
+    torch.cuda.synchronize()
+    oracle.swap_in(k, v, image, dst)
+    assert (as_bits(kd) == k).all() and (as_bits(vd) == v).all()
+    # append: random tokens into random distinct slots of one layer, some entries skipped
+    layer = int(rng.integers(0, layers))
+    B = int(rng.integers(1, 50))
+    slots = rng.permutation(NB * 16)[:B].astype(np.int64)
+    slots[rng.random(B) < 0.2] = -1
+    kn = wl.normal_bf16_np(0, B * Hkv * D, 9300 + seed).reshape(B, Hkv, D)
+    vn = wl.normal_bf16_np(0, B * Hkv * D, 9400 + seed).reshape(B, Hkv, D)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.kv_append(kd[layer], vd[layer], bits_to_torch(kn), bits_to_torch(vn),
+                  torch.from_numpy(slots).cuda(), dev_status=status)
+    torch.cuda.synchronize()
+    oracle.kv_append(k[layer], v[layer], kn, vn, slots)
+    assert int(status.item()) == 0
+    assert (as_bits(kd) == k).all() and (as_bits(vd) == v).all()
