@@ -264,3 +264,25 @@ def test_kv_split_errors():
     assert int(g.status.item()) == api.PA_STATUS_BAD_SEQ_LEN
     assert np.isnan(out[64:]).all()
     assert_parity(out[:64], ref[:64])
+
+
+@pytest.mark.parametrize("scale", [0.0, -0.25])
+@pytest.mark.parametrize("H,Hkv,D", [(8, 2, 128), (8, 8, 64), (4, 1, 256)])
+def test_zero_and_negative_scale(scale, H, Hkv, D):
+    # scale 0: every query is the mean of the V rows it may see; a negative scale turns the
+    # order of the scores around (the kernel's raw-score maximum shortcut needs scale > 0)
+    spec, q, k, v, cu = make_case([300, 64, 17], [300, 10, 17], H, Hkv, D, seed=120)
+    g = GpuPrefill(spec, q, k, v)
+    spec.scale = np.float32(scale)
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, f"scale {scale}")
+    if scale == 0.0:   # closed form, independent of the oracle: running mean of V
+        from helpers import bits_to_torch
+        tab = spec.block_tables[2]
+        vv = bits_to_torch(v).float().cpu().numpy()                      # [NB, Hkv, 16, D]
+        rows = np.stack([vv[tab[t // 16], :, t % 16] for t in range(17)])    # [17, Hkv, D]
+        mean = np.cumsum(rows, axis=0) / np.arange(1, 18)[:, None, None]
+        got = out[int(cu[2]):].reshape(17, Hkv, H // Hkv, D)
+        assert np.abs(got - mean[:, :, None, :]).max() <= 1e-2
