@@ -20,6 +20,11 @@
  *     length or block id) cannot be seen by the host without a sync; they are reported
  *     through the optional `dev_status` word and never make the GPU read outside the pool.
  *   - bf16 is the only element type; accumulation is fp32.
+ *   - Environment variables, each read once per process, for measurements and tests:
+ *     PAGEDKV_PREFILL=mma selects the warp-level-MMA prefill kernel instead of the tcgen05 one;
+ *     PAGEDKV_PREFILL_TILES=1|2 fixes the row tiles per CTA of the tcgen05 prefill kernel;
+ *     PAGEDKV_VARIANT=warps,slots picks another compiled shape of the decode kernel (warps per
+ *     CTA, TMA ring slots per warp; default 8,3).
  */
 #ifndef PAGEDKV_H_
 #define PAGEDKV_H_
