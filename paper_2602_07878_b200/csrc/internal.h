@@ -13,13 +13,13 @@ constexpr int BS = 16;        // tokens per KV block (the only block size suppor
 constexpr int MAX_PART = 512; // largest partition: 32 blocks, one block id per producer lane
 
 // int32 words of the plan header at the start of the workspace
-enum { HDR_N_ITEMS = 0, HDR_N_UNITS = 1, HDR_P = 2, HDR_COUNTER = 3, HDR_STATUS = 4, HDR_WORDS = 64 };
+enum { HDR_N_ITEMS = 0, HDR_N_UNITS = 1, HDR_P = 2, HDR_COUNTER = 3, HDR_STATUS = 4, HDR_N_MULTI = 5, HDR_N_LONG = 6, HDR_WORDS = 64 };
 
 // bit 16 of record.z: the sequence has a single partition, write bf16 output directly
 constexpr int REC_DIRECT = 1 << 16;
 
 struct WsLayout {
-    size_t off_seqinfo, off_records, off_ml, off_o, total;
+    size_t off_seqinfo, off_multi, off_records, off_ml, off_o, total;
     int64_t item_cap;
 };
 // carve a workspace of `bytes` (or compute `total` for `item_cap` when bytes == 0)

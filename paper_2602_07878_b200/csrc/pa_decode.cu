@@ -32,6 +32,8 @@ namespace pk {
 // ======================================================================================
 constexpr int PLAN_THREADS = 1024;
 
+constexpr int COMBINE_LONG = 32;  // rows with more partitions get a whole CTA in the combine
+
 struct PlanParams {
     const int32_t* seq_lens;
     int batch;
@@ -43,6 +45,9 @@ struct PlanParams {
     int total_warps;    // decode warps on the chip
     int* hdr;
     int2* seq_info;     // per sequence: (first partial index, partitions)
+    // the sequences whose rows the combine kernel writes: those with more than COMBINE_LONG
+    // partitions from the front, those with 0 or 2..COMBINE_LONG partitions from the back
+    int* multi;
     int4* records;      // per item: (b, tok0, ntok | flags, partial index)
     int* status;
 };
@@ -60,7 +65,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     __shared__ int s_P, s_bad;
     __shared__ int hist[MAX_PART / BS + 1], start[MAX_PART / BS + 1], cursor[MAX_PART / BS + 1];
     __shared__ int scan_warp[32];
-    __shared__ int s_carry;
+    __shared__ int s_carry, s_multi, s_long;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int max_tok = p.max_blocks * BS;
@@ -83,7 +88,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         if (lane == 0) red[c][warp] = v;
     }
-    if (tid == 0) s_bad = 0;
+    if (tid == 0) s_bad = 0, s_multi = 0, s_long = 0;
     if (tid < MAX_PART / BS + 1) hist[tid] = 0, cursor[tid] = 0;
     __syncthreads();
     if (bad) s_bad = 1;
@@ -113,8 +118,13 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     __syncthreads();
     const int P = s_P;
     if (P == 0) {  // plan does not fit: no work, combine writes zero rows
-        for (int b = tid; b < p.batch; b += PLAN_THREADS) p.seq_info[b] = make_int2(0, 0);
+        for (int b = tid; b < p.batch; b += PLAN_THREADS) {
+            p.seq_info[b] = make_int2(0, 0);
+            p.multi[b] = b;
+        }
         if (tid == 0) {
+            p.hdr[HDR_N_MULTI] = p.batch;
+            p.hdr[HDR_N_LONG] = 0;
             p.hdr[HDR_N_ITEMS] = 0;
             p.hdr[HDR_N_UNITS] = 0;
             p.hdr[HDR_P] = 0;
@@ -133,6 +143,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
             bool dummy = false;
             const int L = clamp_len(p.seq_lens[b], max_tok, dummy);
             np = (L + P - 1) / P;
+            // merged (or zeroed) by the combine kernel
+            if (np > COMBINE_LONG) p.multi[atomicAdd(&s_long, 1)] = b;
+            else if (np != 1) p.multi[p.batch - 1 - atomicAdd(&s_multi, 1)] = b;
             if (np > 0) {
                 if (np > 1) atomicAdd(&hist[full_bin], np - 1);
                 const int last = L - (np - 1) * P;
@@ -170,6 +183,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
             acc += hist[nb];
         }
         p.hdr[HDR_N_ITEMS] = n_items;
+        p.hdr[HDR_N_MULTI] = s_multi;
+        p.hdr[HDR_N_LONG] = s_long;
         p.hdr[HDR_N_UNITS] = n_items * p.Hkv;
         p.hdr[HDR_P] = P;
         p.hdr[HDR_COUNTER] = 3 * p.total_warps;
@@ -431,6 +446,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
 // ======================================================================================
 struct CombineParams {
     const int2* seq_info;
+    const int* multi;  // pa_combine_rows_kernel: the sequences to write
     const float* partial_o;
     const float2* partial_ml;
     __nv_bfloat16* out;
@@ -616,7 +632,8 @@ WsLayout ws_layout(int H, int D, int64_t batch, int64_t item_cap, size_t bytes) 
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
     WsLayout w;
     w.off_seqinfo = up(HDR_WORDS * sizeof(int));
-    w.off_records = w.off_seqinfo + up((size_t)batch * sizeof(int2));
+    w.off_multi = w.off_seqinfo + up((size_t)batch * sizeof(int2));
+    w.off_records = w.off_multi + up((size_t)batch * sizeof(int));
     const size_t per_item = sizeof(int4) + (size_t)H * sizeof(float2) + (size_t)H * D * sizeof(float);
     if (bytes > 0) {
         const size_t fixed = w.off_records + 3 * 256;
@@ -774,6 +791,136 @@ extern "C" int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch,
     return PA_OK;
 }
 
+// The combine of pa_decode itself, over the sequences the plan listed.  A fixed grid of CTAs of
+// eight warps: first the rows of the long sequences (more than COMBINE_LONG partitions), one
+// (sequence, head) row per CTA at a time with warp w taking partitions w, w + 8, ... and the
+// eight sums meeting in shared memory; then the rows of the short ones (2..COMBINE_LONG
+// partitions, or none: a row of zeros), one row per warp, no shared memory, no barrier.  No CTA
+// is spent on rows the attention kernel wrote directly.
+template <int D>
+__global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_constant__ CombineParams p) {
+    constexpr int VPL = D / 32;  // floats per lane
+    constexpr int UB = 8;        // partition rows in flight per warp
+    __shared__ float s_acc[8][D];
+    __shared__ float s_den[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_launch_dependents();
+    pdl_wait();  // partial results of the attention kernel are complete and visible
+    if (blockIdx.x == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
+    const int n_long = p.hdr[HDR_N_LONG] * p.H, n_short = p.hdr[HDR_N_MULTI] * p.H;
+
+    // sum of w_i * (o_i, l_i) over partitions i = start, start + stride, ... < np of one row
+    auto gather = [&](int first, int np, int h, int start, int stride, float M, float (&acc)[VPL],
+                      float& den) {
+        for (int i0 = start; i0 < np; i0 += UB * stride) {
+            float2 ml[UB];
+            float v[UB][VPL];
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const int idx = min(i0 + u * stride, np - 1);
+                ml[u] = p.partial_ml[(size_t)(first + idx) * p.H + h];
+                const float* src = p.partial_o + ((size_t)(first + idx) * p.H + h) * D + lane * VPL;
+                if (VPL >= 4) {
+#pragma unroll
+                    for (int i = 0; i + 3 < VPL; i += 4) {
+                        const float4 x = *reinterpret_cast<const float4*>(src + i);
+                        v[u][i] = x.x, v[u][i + 1] = x.y, v[u][i + 2] = x.z, v[u][i + 3] = x.w;
+                    }
+                } else {
+                    const float2 x = *reinterpret_cast<const float2*>(src);
+                    v[u][0] = x.x, v[u][1] = x.y;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UB; ++u)
+                if (i0 + u * stride < np) {
+                    const float w = ex2(ml[u].x - M);
+                    den += w * ml[u].y;
+#pragma unroll
+                    for (int i = 0; i < VPL; ++i) acc[i] += w * v[u][i];
+                }
+        }
+    };
+    // the row maximum (every lane gets it) and whether a partition was flagged (NaN maximum)
+    auto row_max = [&](int first, int np, int h, bool& bad) -> float {
+        float M = -INFINITY;
+        bad = false;
+        for (int i = lane; i < np; i += 32) {
+            const float m = p.partial_ml[(size_t)(first + i) * p.H + h].x;
+            bad |= m != m;
+            M = fmaxf(M, m);
+        }
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        bad = __any_sync(0xffffffffu, bad);
+        return M == -INFINITY ? 0.f : M;
+    };
+    auto store = [&](__nv_bfloat16* dst, const float (&o)[VPL], bool zero) {
+        if (VPL >= 4) {
+#pragma unroll
+            for (int i = 0; i + 3 < VPL; i += 4) {
+                uint2 x;
+                x.x = zero ? 0u : pack_bf16x2(o[i], o[i + 1]);
+                x.y = zero ? 0u : pack_bf16x2(o[i + 2], o[i + 3]);
+                *reinterpret_cast<uint2*>(dst + i) = x;
+            }
+        } else {
+            *reinterpret_cast<uint32_t*>(dst) = zero ? 0u : pack_bf16x2(o[0], o[1]);
+        }
+    };
+
+    // ---- long rows: one per CTA ----
+    for (int task = blockIdx.x; task < n_long; task += gridDim.x) {
+        const int b = __ldg(&p.multi[task / p.H]), h = task % p.H;
+        const int2 info = p.seq_info[b];
+        bool bad;
+        const float M = row_max(info.x, info.y, h, bad);
+        float acc[VPL];
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
+        float den = 0.f;
+        gather(info.x, info.y, h, warp, 8, M, acc, den);
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) s_acc[warp][lane * VPL + i] = acc[i];
+        if (lane == 0) s_den[warp] = den;
+        __syncthreads();
+        if (warp == 0) {
+            den = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) den += s_den[w];
+            const bool zero = bad || den == 0.f;  // (a flagged row's sums may be NaN)
+            const float inv = zero ? 0.f : 1.f / den;
+            float o[VPL];
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+                float t = 0.f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) t += s_acc[w][lane * VPL + i];
+                o[i] = t * inv;
+            }
+            store(p.out + ((size_t)b * p.H + h) * D + lane * VPL, o, zero);
+        }
+        __syncthreads();
+    }
+    // ---- short rows: one per warp ----
+    const int batch = p.rows / p.H;
+    for (int task = blockIdx.x * 8 + warp; task < n_short; task += gridDim.x * 8) {
+        const int b = __ldg(&p.multi[batch - 1 - task / p.H]), h = task % p.H;
+        const int2 info = p.seq_info[b];
+        bool bad;
+        const float M = row_max(info.x, info.y, h, bad);
+        float acc[VPL];
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
+        float den = 0.f;
+        gather(info.x, info.y, h, 0, 1, M, acc, den);
+        const bool zero = info.y == 0 || bad || den == 0.f;
+        const float inv = zero ? 0.f : 1.f / den;
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) acc[i] *= inv;
+        store(p.out + ((size_t)b * p.H + h) * D + lane * VPL, acc, zero);
+    }
+}
+
 template <int MODE>
 static cudaError_t launch_combine(int D, int grid, cudaStream_t st, const CombineParams& cp) {
     return D == 256   ? launch_pdl(pa_combine_kernel<256, MODE>, dim3(grid), dim3(128), 0, st, cp)
@@ -859,6 +1006,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
         pp.total_warps = total_warps;
         pp.hdr = hdr;
         pp.seq_info = reinterpret_cast<int2*>(ws + w.off_seqinfo);
+        pp.multi = reinterpret_cast<int*>(ws + w.off_multi);
         pp.records = reinterpret_cast<int4*>(ws + w.off_records);
         pp.status = status;
         count_launch();
@@ -873,6 +1021,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
 
     CombineParams cp = {};
     cp.seq_info = reinterpret_cast<const int2*>(ws + w.off_seqinfo);
+    cp.multi = reinterpret_cast<const int*>(ws + w.off_multi);
     cp.partial_o = dp.partial_o;
     cp.partial_ml = dp.partial_ml;
     cp.out = dp.out;
@@ -886,8 +1035,11 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     }
     const int cgrid = cp.rows;
     count_launch();
-    rc = check_cuda(part ? launch_combine<COMBINE_TO_PARTIAL>(D, cgrid, st, cp)
-                         : launch_combine<COMBINE_FINAL>(D, cgrid, st, cp));
+    const dim3 rgrid(8 * dev.sm_count), rblock(256);  // every SM full of warps with loads in flight
+    rc = check_cuda(part       ? launch_combine<COMBINE_TO_PARTIAL>(D, cgrid, st, cp)
+                    : D == 256 ? launch_pdl(pa_combine_rows_kernel<256>, rgrid, rblock, 0, st, cp)
+                    : D == 128 ? launch_pdl(pa_combine_rows_kernel<128>, rgrid, rblock, 0, st, cp)
+                               : launch_pdl(pa_combine_rows_kernel<64>, rgrid, rblock, 0, st, cp));
     if (prof) cudaEventRecord(prof_ev.ev[3], st);
     return rc;
 }
