@@ -255,6 +255,11 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
     const int g = lane >> 2, t = lane & 3;
     const uint32_t slots = base + warp * (NSLOT * SLOT);
     const uint32_t bars = base + NW * NSLOT * SLOT + warp * (NSLOT * 8);
+    // Head_dim 256: the output accumulator alone takes 128 registers per thread, so the Q
+    // fragments of the next unit are parked in shared memory (one word per lane and fragment)
+    // instead of in a second set of registers, and fetched when that unit becomes current.
+    constexpr bool QSTASH = D == 256;
+    const uint32_t stash = base + NW * NSLOT * SLOT + NW * NSLOT * 8 + warp * (KS * QW * 128) + lane * 4;
 
     if (lane == 0) {
 #pragma unroll
@@ -284,7 +289,11 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             rec = __ldg(&p.records[item]);
         }
     };
-    auto build = [&](const int4& rec, int kvh, bool valid, Unit& u) {
+    auto st_stash = [&](int ks, int i, uint32_t v) {
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stash + (ks * QW + i) * 128), "r"(v) : "memory");
+    };
+    // `parked`: the fragments go to the stash (head_dim 256, the unit after the current one)
+    auto build = [&](const int4& rec, int kvh, bool valid, Unit& u, bool parked) {
         u.valid = valid;
         u.b = rec.x;
         u.tok0 = rec.y;
@@ -295,29 +304,34 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         u.nblk = (u.ntok + BS - 1) / BS;
         u.bad = false;
         u.id = 0;
-        if (valid) {
-            if (lane < u.nblk)
-                u.id = __ldg(&p.block_tables[(size_t)u.b * p.max_blocks + u.tok0 / BS + lane]);
-            const size_t row0 = ((size_t)u.b * H + (size_t)kvh * G) * D;
+        if (valid && lane < u.nblk)
+            u.id = __ldg(&p.block_tables[(size_t)u.b * p.max_blocks + u.tok0 / BS + lane]);
+        const size_t row0 = valid ? ((size_t)u.b * H + (size_t)kvh * G) * D : 0;
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                // a0: (row g, k 2t..), a2: (row g, k 8+2t..); a1/a3 the same for row g+8
-                const size_t c = ks * 16 + 2 * t;
-                u.qa[ks][0] = g < G ? __ldg(&q32[(row0 + (size_t)g * D + c) >> 1]) : 0u;
-                u.qa[ks][QW == 4 ? 2 : 1] =
-                    g < G ? __ldg(&q32[(row0 + (size_t)g * D + c + 8) >> 1]) : 0u;
-                if (HI) {
-                    u.qa[ks][1] = g + 8 < G ? __ldg(&q32[(row0 + (size_t)(g + 8) * D + c) >> 1]) : 0u;
-                    u.qa[ks][QW - 1] =
-                        g + 8 < G ? __ldg(&q32[(row0 + (size_t)(g + 8) * D + c + 8) >> 1]) : 0u;
-                }
+        for (int ks = 0; ks < KS; ++ks) {
+            // a0: (row g, k 2t..), a2: (row g, k 8+2t..); a1/a3 the same for row g+8
+            const size_t c = ks * 16 + 2 * t;
+            uint32_t w[QW];
+            w[0] = valid && g < G ? __ldg(&q32[(row0 + (size_t)g * D + c) >> 1]) : 0u;
+            w[QW == 4 ? 2 : 1] = valid && g < G ? __ldg(&q32[(row0 + (size_t)g * D + c + 8) >> 1]) : 0u;
+            if (HI) {
+                w[1] = valid && g + 8 < G ? __ldg(&q32[(row0 + (size_t)(g + 8) * D + c) >> 1]) : 0u;
+                w[QW - 1] =
+                    valid && g + 8 < G ? __ldg(&q32[(row0 + (size_t)(g + 8) * D + c + 8) >> 1]) : 0u;
             }
-        } else {
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks)
-#pragma unroll
-                for (int i = 0; i < QW; ++i) u.qa[ks][i] = 0u;
+            for (int i = 0; i < QW; ++i) {
+                if (QSTASH && parked) st_stash(ks, i, w[i]);
+                else u.qa[ks][i] = w[i];
+            }
         }
+    };
+    auto unpark = [&](Unit& u) {  // the parked fragments of the unit that has become current
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int i = 0; i < QW; ++i)
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(u.qa[ks][i]) : "r"(stash + (ks * QW + i) * 128));
     };
 
     Unit U0, U1;
@@ -333,8 +347,8 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         load_record(gw + total_warps, r1, k1, v1);
         load_record(gw + 2 * total_warps, recB, kvhB, validB);
         if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
-        build(r0, k0, v0, U0);
-        build(r1, k1, v1, U1);
+        build(r0, k0, v0, U0, false);
+        build(r1, k1, v1, U1, true);
     }
 
     AttnFrag<D, HI> A;
@@ -430,7 +444,8 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             }
             // advance the fetch pipeline
             U0 = U1;
-            build(recB, kvhB, validB, U1);
+            if (QSTASH) unpark(U0);
+            build(recB, kvhB, validB, U1, true);
             const int w = __shfl_sync(0xffffffffu, wraw, 0);
             load_record(w, recB, kvhB, validB);
             if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
@@ -672,7 +687,9 @@ template <int D, bool HI, int NW, int NSLOT>
 static int launch_decode(const CUtensorMap& km, const CUtensorMap& vm, const DecodeParams& dp,
                          const DeviceInfo& dev, int* grid_out, bool launch, cudaStream_t st) {
     auto kern = pa_decode_kernel<D, HI, NW, NSLOT>;
-    const int smem = NW * NSLOT * (2 * BS * D * 2) + NW * NSLOT * 8 + 1024;
+    // at head_dim 256 the Q fragments of the unit after the current one wait in shared memory
+    const int stash = D == 256 ? NW * (D / 16) * (HI ? 4 : 2) * 32 * 4 : 0;
+    const int smem = NW * NSLOT * (2 * BS * D * 2) + NW * NSLOT * 8 + stash + 1024;
     if (smem > dev.smem_optin) return PA_ERR_SHAPE;
     static int configured_dev = -1, ctas_per_sm = 0;
     static std::mutex mu;
