@@ -323,6 +323,12 @@ def run_ours(args):
     dev = "cuda"
 
     spec = wl.config_spec(args.workload)
+    if args.decode_shape:
+        # the workload's lengths and pool occupancy with another layer shape (H, Hkv, D)
+        hq, hkv, hd = (int(x) for x in args.decode_shape.split(","))
+        spec = wl.make_spec(f"{spec.name}_h{hq}_kv{hkv}_d{hd}", seq_lens=spec.seq_lens,
+                            num_q_heads=hq, num_kv_heads=hkv, head_dim=hd,
+                            num_blocks=spec.num_blocks, seed=spec.seed)
     q = wl.q_torch(spec, dev)
     k, v = wl.pools_torch(spec, dev)
     tables = torch.from_numpy(spec.block_tables).to(dev)
@@ -986,6 +992,9 @@ def main():
     ap.add_argument("--no-recompute", action="store_true")
     ap.add_argument("--recompute-chunk", type=int, default=512,
                     help="query tokens per pa_prefill call of the recompute leg")
+    ap.add_argument("--decode-shape", default="",
+                    help="H,Hkv,D of the decode legs when they should differ from the workload's "
+                         "(e.g. 16,8,256); lengths and occupancy stay the workload's")
     ap.add_argument("--recompute-shape", default="",
                     help="H,Hkv,D of the recompute leg when it should differ from the workload's "
                          "(e.g. 16,8,256)")
