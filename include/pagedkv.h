@@ -247,7 +247,8 @@ int pa_prefill_workspace_bytes(int32_t max_batch, size_t* bytes);
  *   dev_status    as for pa_decode: inconsistent lengths set PA_STATUS_BAD_SEQ_LEN (that
  *                 sequence's rows are left unwritten), a bad used block id sets
  *                 PA_STATUS_BAD_BLOCK_ID (affected rows are zero)
- * Two kernels are enqueued (a one-CTA plan and the attention kernel).
+ * One or two kernels are enqueued (the attention kernel; before it a one-CTA plan when the
+ * batch has more than 32 sequences or the warp-level kernel runs).
  */
 int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const void* v_cache,
                const int32_t* block_tables, int32_t max_blocks_per_seq, const int32_t* ctx_lens,
@@ -272,7 +273,7 @@ int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const 
  *                     used up to what pa_prefill_split_workspace_bytes(shape, batch, total_q,
  *                     splits) says fits.
  * pa_prefill is this call with kv_split_tokens = 0.
- * Two or three kernels are enqueued.  Errors as for pa_prefill; a split that met a bad
+ * One to three kernels are enqueued (plan, attention, merge).  Errors as for pa_prefill; a split that met a bad
  * block id zeroes the rows that depend on it.
  */
 int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t max_batch,

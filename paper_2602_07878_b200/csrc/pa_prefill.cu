@@ -338,6 +338,9 @@ struct PrefillTcParams {
     int split_steps, split_cap;
     float* part_ml;
     float* part_o;
+    // Batches of at most 32 sequences need no plan kernel: every CTA validates the lengths and
+    // scans the unit counts itself (one warp, a few hundred cycles) and only CTA 0 reports.
+    int fold_plan, total_q;
 };
 
 template <int D, int NT>
@@ -368,19 +371,46 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
 
     // ---- which tile -------------------------------------------------------------------------
     const int G = p.G, H = p.H, Hkv = p.Hkv, tpt = tp.tokens_per_tile;
-    const int n_units = p.hdr[PF_N_GROUPS] * Hkv;
+    __shared__ int s_gstart[33];
+    const int* gs = p.gstart;
+    if (tp.fold_plan) {  // the plan kernel's work for a small batch (same checks, same counts)
+        if (warp == 0) {
+            int n = 0;
+            bool bad = false;
+            if (lane < p.batch) {
+                const int q0 = p.cu_q_lens[lane], q1 = p.cu_q_lens[lane + 1], L = p.ctx_lens[lane];
+                const int ql = q1 - q0;
+                const bool ok = q0 >= 0 && ql >= 0 && q1 <= tp.total_q && L >= ql &&
+                                L <= p.max_blocks * BS && (lane > 0 || q0 == 0);
+                bad = !ok;
+                n = ok ? (ql + p.tpg - 1) / p.tpg * kv_splits(L, tp.split_steps) : 0;
+            }
+            int incl = n;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            s_gstart[lane + 1] = incl;
+            if (lane == 0) s_gstart[0] = 0;
+            if (blockIdx.x == 0 && __any_sync(0xffffffffu, bad) && lane == 0)
+                atomicOr(p.status, PA_STATUS_BAD_SEQ_LEN);
+        }
+        __syncthreads();
+        gs = s_gstart;
+    }
+    const int n_units = (tp.fold_plan ? s_gstart[p.batch] : p.hdr[PF_N_GROUPS]) * Hkv;
     if ((int)blockIdx.x >= n_units) return;
     const int u = n_units - 1 - blockIdx.x;  // later tiles see more tokens: start them first
     const int gi = u / Hkv, kvh = u - gi * Hkv;
     int lo = 0, hi = p.batch;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (p.gstart[mid] <= gi) lo = mid; else hi = mid;
+        if (gs[mid] <= gi) lo = mid; else hi = mid;
     }
     const int b = lo;
     const int q0 = p.cu_q_lens[b], ql = p.cu_q_lens[b + 1] - q0, L = p.ctx_lens[b];
     const int n_split = kv_splits(L, tp.split_steps);   // units per row group of this sequence
-    const int r = gi - p.gstart[b];
+    const int r = gi - gs[b];
     const int split = r % n_split;
     const int tok0 = (r / n_split) * (NT * tpt);        // first query token of the CTA
     const int ntok_cta = min(NT * tpt, ql - tok0);
@@ -1108,7 +1138,8 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
     plan.hdr = hdr;
     plan.gstart = hdr + PF_WORDS;
     plan.status = dev_status ? dev_status : hdr + PF_STATUS;
-    {
+    const bool fold_plan = use_tc && batch <= 32;  // the attention CTAs plan for themselves
+    if (!fold_plan) {
         // launched as a programmatic dependent of whatever precedes it in the stream (the
         // previous chunk's merge): its launch latency hides under that kernel's tail
         cudaLaunchConfig_t cfg = {};
@@ -1151,6 +1182,8 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
         tp.tokens_per_tile = 128 / G;
         tp.split_steps = ts.split_steps;
         tp.split_cap = ts.split_cap;
+        tp.fold_plan = fold_plan ? 1 : 0;
+        tp.total_q = total_q;
         tp.part_ml = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + base_bytes);
         tp.part_o = tp.part_ml + (size_t)total_q * H * ts.split_cap * 2;
         const int64_t max_ctas = ((int64_t)total_q / plan.tpg + batch) * pp.Hkv * ts.split_cap;

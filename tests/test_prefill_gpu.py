@@ -286,3 +286,25 @@ def test_zero_and_negative_scale(scale, H, Hkv, D):
         mean = np.cumsum(rows, axis=0) / np.arange(1, 18)[:, None, None]
         got = out[int(cu[2]):].reshape(17, Hkv, H // Hkv, D)
         assert np.abs(got - mean[:, :, None, :]).max() <= 1e-2
+
+
+@pytest.mark.parametrize("n_seq", [32, 33, 70])
+def test_batches_around_32_sequences(n_seq):
+    # up to 32 sequences the attention CTAs plan for themselves; beyond that a plan kernel runs
+    rng = np.random.default_rng(n_seq)
+    ctx = [int(x) for x in rng.integers(1, 200, n_seq)]
+    qlens = [int(rng.integers(0, c + 1)) for c in ctx]
+    qlens[0] = max(qlens[0], 1)
+    spec, q, k, v, cu = make_case(ctx, qlens, 8, 2, 128, seed=200 + n_seq)
+    g = GpuPrefill(spec, q, k, v)
+    n0 = api.pa_launch_count()
+    out = torch_to_f64(g.run(spec.seq_lens, cu))
+    assert api.pa_launch_count() - n0 == (1 if n_seq <= 32 else 2)
+    ref = oracle.pa_prefill(q, k, v, spec.block_tables, spec.seq_lens, cu, spec.scale)
+    assert int(g.status.item()) == 0
+    assert_parity(out, ref, f"{n_seq} sequences")
+    # and a refused sequence is reported either way
+    bad_ctx = spec.seq_lens.copy()
+    bad_ctx[n_seq - 1] = -3
+    g.run(bad_ctx, cu)
+    assert int(g.status.item()) == api.PA_STATUS_BAD_SEQ_LEN
