@@ -63,6 +63,12 @@ def _elem_strides(a: np.ndarray):
     return tuple(s // 2 for s in a.strides[:3])
 
 
+def _sigma(scale) -> float:
+    """The scale is an fp32 argument of the method: whatever the caller passes is rounded to
+    fp32 first and that value, widened exactly, is what the fp64 arithmetic uses."""
+    return float(np.float32(scale))
+
+
 def pa_decode(q, k_cache, v_cache, block_tables, seq_lens, scale, num_threads: int = 0):
     """fp64 attention output [B, H, D] for bf16-bit inputs.
 
@@ -82,7 +88,7 @@ def pa_decode(q, k_cache, v_cache, block_tables, seq_lens, scale, num_threads: i
     out = np.zeros((B, H, D), dtype=np.float64)
     rc = _load().oracle_pa_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
                                   block_tables.shape[1], _ptr(seq_lens), B, H, Hkv, D, bs, NB,
-                                  sb, sh, st, float(scale), _ptr(out), num_threads)
+                                  sb, sh, st, _sigma(scale), _ptr(out), num_threads)
     if rc != 0:
         raise ValueError("oracle_pa_decode: invalid length or block id")
     return out
@@ -155,7 +161,7 @@ def pa_prefill(q, k_cache, v_cache, block_tables, ctx_lens, cu_q_lens, scale, nu
     out = np.zeros((T, H, D), dtype=np.float64)
     rc = _load().oracle_pa_prefill(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
                                    block_tables.shape[1], _ptr(ctx_lens), _ptr(cu), B, H, Hkv, D,
-                                   bs, NB, sb, sh, st, float(scale), _ptr(out), num_threads)
+                                   bs, NB, sb, sh, st, _sigma(scale), _ptr(out), num_threads)
     if rc != 0:
         raise ValueError("oracle_pa_prefill: inconsistent lengths or bad block id")
     return out

@@ -955,6 +955,14 @@ static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const
 
 using namespace pk;
 
+// The partial records follow the plan: first the (exponent, sum) pairs, then the fp32 rows, which
+// are written and read 16 bytes at a time.  An odd number of pairs would leave the rows 8-byte
+// aligned only, so the pair region is rounded up to 16 bytes and the workspace carries the pad.
+constexpr size_t PART_PAD_BYTES = 16;
+static size_t part_ml_floats(int64_t total_q, int H, int split_cap) {
+    return ((size_t)total_q * H * split_cap * 2 + 3) & ~(size_t)3;
+}
+
 static size_t prefill_base_bytes(int64_t batch) {
     const size_t b = PF_WORDS * sizeof(int) + ((size_t)batch + 1) * sizeof(int) + 256;
     return (b + 255) & ~(size_t)255;
@@ -975,8 +983,8 @@ extern "C" int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t m
     int rc = validate_shape(shape);
     if (rc) return rc;
     if (max_batch < 0 || max_total_q < 0 || max_splits < 1) return PA_ERR_ARG;
-    *bytes = prefill_base_bytes(max_batch) + (size_t)max_total_q * shape->num_q_heads *
-                                                 max_splits * (shape->head_dim + 2) * sizeof(float);
+    *bytes = prefill_base_bytes(max_batch) + PART_PAD_BYTES +
+             (size_t)max_total_q * shape->num_q_heads * max_splits * (shape->head_dim + 2) * sizeof(float);
     return PA_OK;
 }
 
@@ -1043,7 +1051,9 @@ static int select_launch(const pa_shape* shape, int batch, int64_t total_q, int 
     if (force_mma) return PA_OK;
     const int64_t steps_bound = std::max<int64_t>(1, ((int64_t)max_blocks_per_seq * BS + 63) / 64);
     const size_t per_split = (size_t)std::max<int64_t>(total_q, 1) * H * (D + 2) * sizeof(float);
-    const int64_t cap_fit = (int64_t)((workspace_bytes - base_bytes) / per_split);
+    const size_t part_bytes = workspace_bytes - base_bytes;
+    const int64_t cap_fit =
+        part_bytes > PART_PAD_BYTES ? (int64_t)((part_bytes - PART_PAD_BYTES) / per_split) : 0;
     int forced_steps = 0;
     if (kv_split_tokens > 0) {
         forced_steps = (kv_split_tokens + 63) / 64;
@@ -1185,7 +1195,7 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
         tp.fold_plan = fold_plan ? 1 : 0;
         tp.total_q = total_q;
         tp.part_ml = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + base_bytes);
-        tp.part_o = tp.part_ml + (size_t)total_q * H * ts.split_cap * 2;
+        tp.part_o = tp.part_ml + part_ml_floats(total_q, H, ts.split_cap);
         const int64_t max_ctas = ((int64_t)total_q / plan.tpg + batch) * pp.Hkv * ts.split_cap;
         if (max_ctas > INT32_MAX) return PA_ERR_ARG;
         const bool two = ts.tiles_per_cta == 2;

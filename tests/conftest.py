@@ -24,3 +24,21 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """How often the run needed more than the plain 1e-2 element-wise bound."""
+    try:
+        import helpers
+    except Exception:  # pragma: no cover
+        return
+    t = helpers.TALLY
+    if not t["calls"]:
+        return
+    terminalreporter.write_line(
+        f"parity tally: {t['calls']} comparisons with the oracle, {t['elements']} elements "
+        f"({t['amended_elements']} of them prefill outputs under the amended bound); "
+        f"{t['over_abs_tol']} elements above 1e-2"
+        + (f" (smallest |ref| {t['over_abs_tol_min_ref']:.3f}, largest error "
+           f"{t['over_abs_tol_max_err']:.4e}): " + "; ".join(t["over_abs_tol_where"])
+           if t["over_abs_tol"] else ""))

@@ -7,26 +7,83 @@ import oracle
 from paper_2602_07878_b200 import api
 from paper_2602_07878_b200 import workloads as wl
 
-# Tolerance for bf16 inputs with fp32 accumulation: element-wise |gpu - ref| <= 1e-2 and,
-# per (sequence, head) row, max_d |gpu - ref| <= 2e-2 * max_d |ref|.  The output is bf16:
-# from 2 upwards its values are 2^-6 apart (2^-5 from 4), so rounding the result alone takes
-# up to 7.8e-3 (1.6e-2) and the bf16 rounding of the softmax weights adds up to 2^-9 of the
-# magnitude; there the element-wise bound is one spacing of bf16 at |ref| instead of 1e-2.
-# Outputs that large need a softmax that is nearly one-hot on an extreme element of V.
+# Tolerance.  Decode (pa_decode and every entry point built on it): the stated one for bf16
+# inputs with fp32 accumulation -- element-wise |gpu - ref| <= 1e-2 and, per (sequence, head)
+# row, max_d |gpu - ref| <= 2e-2 * max_d |ref| -- with no exception.
+#
+# Prefill (pa_prefill, pa_prefill_split) has no stated tolerance of its own; its bound follows
+# from its arithmetic and equals the decode bound except on rare elements.  With w_t the softmax
+# weights of a row, the kernel computes sum_t bf16(w_t) V_t (the weights are a tensor-core operand)
+# over a row sum of the unrounded weights, then rounds the result to bf16:
+#     |gpu - ref|  <=  half a bf16 spacing at |ref|        (rounding of the result)
+#                    + 2^-8 * sum_t w_t |V_t|               (rounding of each weight)
+#                    + 1e-3                                 (fp32 sums, approximated exponentials)
+# bf16 keeps 8 significant bits, so rounding to it moves a value by up to 2^-8 of itself (the
+# unit roundoff; half a spacing is 2^-8 of the power of two below the value).  The middle term
+# is the attention output over |V| and comes from the same oracle.  Where that total exceeds
+# 1e-2 it replaces 1e-2 (`amended`): a row whose softmax is one-hot on an element of V of
+# magnitude 2.5 may be off by 7.8e-3 + 9.8e-3.  It takes an output of magnitude above 1, i.e. a
+# softmax concentrated on a few extreme elements of V, for the total to pass 1e-2.  The tally
+# below counts the elements that ever use it.  The row-normalised 2e-2 bound is the same for
+# both.
 ABS_TOL = 1e-2
 REL_TOL = 2e-2
 GUARD = 4096            # guard elements on each side of a test's output buffer
 GUARD_BITS = 0x7A5A     # their content (int16 view)
 
+# running totals over every assert_parity call of the process (printed at the end of the run)
+TALLY = {"calls": 0, "elements": 0, "amended_calls": 0, "amended_elements": 0,
+         "over_abs_tol": 0, "over_abs_tol_min_ref": float("inf"), "over_abs_tol_max_err": 0.0,
+         "over_abs_tol_where": []}
 
-def assert_parity(gpu: np.ndarray, ref: np.ndarray, what: str = "", abs_tol: float = ABS_TOL):
+
+def amended_bound(ref: np.ndarray, abs_ref: np.ndarray) -> np.ndarray:
+    """Element-wise prefill bound: max(1e-2, half spacing at |ref| + 2^-8 abs_ref + 1e-3), where
+    abs_ref is the oracle's output for the same inputs with V replaced by |V|."""
+    a = np.abs(ref)
+    half_spacing = 2.0 ** (np.floor(np.log2(np.maximum(a, 1e-30))) - 8)   # bf16: 8 significant bits
+    return np.maximum(ABS_TOL, half_spacing + abs_ref * 2.0 ** -8 + 1e-3)
+
+
+def abs_bits(v_bits: np.ndarray) -> np.ndarray:
+    """|V| on bf16 bit patterns (sign bit cleared; NaN tails stay NaN and stay masked)."""
+    return v_bits & np.uint16(0x7FFF)
+
+
+def prefill_ref(q, k, v, tables, ctx, cu, scale):
+    """(oracle output, thunk returning the oracle output over |V|) for a prefill comparison."""
+    ref = oracle.pa_prefill(q, k, v, tables, ctx, cu, scale)
+    return ref, (lambda: oracle.pa_prefill(q, k, abs_bits(v), tables, ctx, cu, scale))
+
+
+def assert_parity(gpu: np.ndarray, ref: np.ndarray, what: str = "", abs_tol: float = ABS_TOL,
+                  amended=None):
+    """Compare a GPU result with the oracle.  `amended` (prefill results only) is a callable
+    returning the oracle's output over |V|, shaped like `ref`; it is evaluated only when some
+    element exceeds the plain bound."""
     gpu = np.asarray(gpu, dtype=np.float64)
     assert gpu.shape == ref.shape, (gpu.shape, ref.shape)
     assert np.isfinite(gpu).all(), f"{what}: non-finite output"
     err = np.abs(gpu - ref)
-    spacing = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7)   # of bf16 at |ref|
-    excess = err - np.maximum(abs_tol, np.where(np.abs(ref) >= 2.0, spacing, 0.0))
-    assert excess.max(initial=-1.0) <= 0.0, f"{what}: abs err {err.max():.3e}"
+    bound = np.full_like(err, abs_tol)
+    over = err > ABS_TOL
+    TALLY["calls"] += 1
+    TALLY["elements"] += err.size
+    if amended is not None:
+        TALLY["amended_calls"] += 1
+        TALLY["amended_elements"] += err.size
+    if over.any():
+        TALLY["over_abs_tol"] += int(over.sum())
+        TALLY["over_abs_tol_min_ref"] = min(TALLY["over_abs_tol_min_ref"], float(np.abs(ref[over]).min()))
+        TALLY["over_abs_tol_max_err"] = max(TALLY["over_abs_tol_max_err"], float(err[over].max()))
+        TALLY["over_abs_tol_where"].append(f"{what}: {int(over.sum())} of {err.size}")
+        if amended is not None:
+            abs_ref = np.asarray(amended(), dtype=np.float64)
+            assert abs_ref.shape == ref.shape
+            bound = amended_bound(ref, abs_ref)
+    worst = np.unravel_index(np.argmax(err - bound), err.shape) if err.size else ()
+    assert (err <= bound).all(), (f"{what}: abs err {err[worst]:.3e} at ref {ref[worst]:.4f} "
+                                  f"(bound {bound[worst]:.3e})")
     row_err = err.reshape(-1, err.shape[-1]).max(axis=1)
     row_ref = np.abs(ref).reshape(-1, ref.shape[-1]).max(axis=1)
     rel = row_err / np.maximum(row_ref, 1e-30)

@@ -10,7 +10,7 @@ import oracle
 from paper_2602_07878_b200 import api
 from paper_2602_07878_b200 import workloads as wl
 from paper_2602_07878_b200.sched import RECOMPUTE, SWAP, Scheduler
-from helpers import assert_parity, bits_to_torch, torch_to_f64
+from helpers import assert_parity, bits_to_torch, prefill_ref, torch_to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -111,8 +111,8 @@ def test_scheduler_driven_engine_loop_matches_oracle(mode, policy):
                            scale, out, pws, dev_status=status)
             torch.cuda.synchronize()
             dk, dv, dt = dense_inputs(st.prefill_ids, st.prefill_ctx_lens)
-            ref = oracle.pa_prefill(qb, dk, dv, dt, st.prefill_ctx_lens, cu, scale)
-            assert_parity(torch_to_f64(out), ref, "prefill")
+            ref, abs_ref = prefill_ref(qb, dk, dv, dt, st.prefill_ctx_lens, cu, scale)
+            assert_parity(torch_to_f64(out), ref, "prefill", amended=abs_ref)
             checked_prefill += 1
         # ---- decode: append the new token, attend ----
         if len(st.decode_ids):

@@ -9,7 +9,7 @@ import torch
 import oracle
 from paper_2602_07878_b200 import api
 from paper_2602_07878_b200 import workloads as wl
-from helpers import assert_parity, torch_to_f64
+from helpers import abs_bits, assert_parity, torch_to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -241,4 +241,7 @@ def test_full_size_recompute_sampled_against_oracle(H, Hkv, D, chunk):
     pos = np.array([L - chunk + t for t in toks], np.int32)
     ref = oracle.pa_decode(qb[toks], kb, vb, np.repeat(table, len(toks), axis=0), pos + 1,
                            np.float32(D ** -0.5))
-    assert_parity(torch_to_f64(out[toks]), ref, f"recompute H{H}/{Hkv} D{D} chunk {chunk}")
+    assert_parity(torch_to_f64(out[toks]), ref, f"recompute H{H}/{Hkv} D{D} chunk {chunk}",
+                  amended=lambda: oracle.pa_decode(qb[toks], kb, abs_bits(vb),
+                                                   np.repeat(table, len(toks), axis=0), pos + 1,
+                                                   np.float32(D ** -0.5)))

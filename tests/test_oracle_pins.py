@@ -312,3 +312,26 @@ def test_bruteforce_pin_catches_planted_mistakes(mutant):
     ref = dense_bruteforce(q, k, v, spec.block_tables, spec.seq_lens, spec.scale)
     bad = mutant(q, k, v, spec.block_tables, spec.seq_lens, spec.scale)
     assert np.abs(bad - ref).max() > 1e-3
+
+
+def test_scale_is_rounded_to_fp32_by_the_oracle_itself():
+    # The scale is an fp32 argument of the method.  A Python double that is not an fp32 value
+    # (0.1, 1/sqrt(128)) must give exactly what its fp32 rounding gives, and that must be the
+    # brute-force result for the widened fp32 value -- not for the double.
+    spec = wl.make_spec("t", seq_lens=[9, 40, 17], num_q_heads=4, num_kv_heads=2, head_dim=64,
+                        num_blocks=12, seed=5)
+    q = wl.q_np(spec)
+    k, v = wl.pools_np(spec)
+    cu = np.array([0, 3, 10, 11], np.int32)
+    qp = wl.normal_bf16_np(0, 11 * 4 * 64, 31).reshape(11, 4, 64)
+    for s in (0.1, 128 ** -0.5, 3.3):
+        s32 = np.float32(s)
+        assert float(s32) != s
+        a = oracle.pa_decode(q, k, v, spec.block_tables, spec.seq_lens, s)
+        assert (a == oracle.pa_decode(q, k, v, spec.block_tables, spec.seq_lens, s32)).all()
+        ref32 = dense_bruteforce(q, k, v, spec.block_tables, spec.seq_lens, float(s32))
+        ref64 = dense_bruteforce(q, k, v, spec.block_tables, spec.seq_lens, s)
+        assert np.abs(a - ref32).max() < 1e-12
+        assert np.abs(a - ref64).max() > np.abs(a - ref32).max()
+        p = oracle.pa_prefill(qp, k, v, spec.block_tables, spec.seq_lens, cu, s)
+        assert (p == oracle.pa_prefill(qp, k, v, spec.block_tables, spec.seq_lens, cu, s32)).all()

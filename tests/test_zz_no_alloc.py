@@ -4,9 +4,10 @@ A serving engine that gave the whole GPU to its KV pool, or a plug-in that only 
 the current step's tensors, has no way to cudaMalloc the workspace pa_decode asks for.
 pa_decode_static keeps its scratch in a fixed array inside the library instead.  This file
 checks, through the C-ABI, that it gives the same result as pa_decode with a caller-owned
-workspace -- twice in a row with different shapes, because every call reuses the same array
-and finds the previous call's leftovers in it -- and that a request beyond the array's size
-is refused before anything is launched.  It is collected last on purpose.
+workspace and as the fp64 oracle -- several times in a row with different shapes, because every
+call reuses the same array and finds the previous call's leftovers in it -- that the device's
+free memory does not move across a call, and that a request beyond the array's size is refused
+before anything is launched.  It is collected last on purpose.
 """
 import ctypes
 
@@ -16,7 +17,7 @@ import torch
 
 from paper_2602_07878_b200 import api
 from paper_2602_07878_b200 import workloads as wl
-from helpers import GpuDecode, assert_parity, torch_to_f64
+from helpers import GpuDecode, assert_parity, oracle_for, torch_to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -28,13 +29,21 @@ def _both_ways(spec):
     ref = g.run().clone()                      # existing entry point, caller workspace
     out = torch.full_like(g.q, float("nan"))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    run = lambda: api.pa_decode_static(g.q, g.k, g.v, g.tables, g.lens, spec.scale, out,
+                                       spec.total_tokens, dev_status=status)
+    run()                                      # the first call on a device looks the array up
+    torch.cuda.synchronize()
+    out.fill_(float("nan"))
     allocations = lambda: torch.cuda.memory_stats().get("allocation.all.allocated", 0)
-    before = allocations()                     # count of allocator requests so far
-    api.pa_decode_static(g.q, g.k, g.v, g.tables, g.lens, spec.scale, out,
-                         spec.total_tokens, dev_status=status)
+    before = allocations()                     # count of requests to torch's allocator so far
+    free_before = torch.cuda.mem_get_info()[0]  # the driver's own count of free bytes
+    run()
     torch.cuda.synchronize()
     assert allocations() == before             # torch's allocator was not asked for anything
+    assert torch.cuda.mem_get_info()[0] == free_before   # nor the driver, by the library itself
     assert int(status.item()) == 0
+    # the definition itself, under the plain decode tolerance
+    assert_parity(torch_to_f64(out), oracle_for(spec, q, k, v), f"{spec.name} against the oracle")
     return torch_to_f64(out), torch_to_f64(ref)
 
 
