@@ -91,8 +91,8 @@ typedef struct kv_pool_desc {
  * Bytes of device workspace pa_decode needs for batches of at most `max_batch` sequences
  * holding at most `max_total_tokens` cached tokens in total.  `partition_tokens` is the
  * value that will be passed to pa_decode (0 = automatic).  The workspace holds the
- * partition plan and the fp32 partial results of sequences that are split (a2-a4 of the
- * decode path: plan, partition attention, combine).
+ * partition plan and the fp32 partial results of sequences that are split (it serves the three
+ * stages of a call: plan, partition attention, combine).
  */
 int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch, int64_t max_total_tokens,
                        int32_t partition_tokens, size_t* bytes);
@@ -130,6 +130,25 @@ int pa_decode(const pa_shape* shape, const void* q, const void* k_cache, const v
               const int32_t* block_tables, int32_t max_blocks_per_seq, const int32_t* seq_lens,
               int32_t batch, float scale, void* out, void* workspace, size_t workspace_bytes,
               int32_t partition_tokens, int32_t flags, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * pa_decode whose q and out are views into wider tensors (the same step of Section 2.1 / 2.2).
+ * Tensor-parallel serving (Section 6.4: TP 2/4/8) gives each GPU a slice of the KV heads and the
+ * query heads of their groups; an engine that keeps a batch-wide [batch, H_all, D] tensor, or
+ * takes q straight out of a fused QKV projection, then holds this rank's heads as a strided view.
+ * Row (b, h) of q starts at q + b * q_stride_seq + h * D elements, row (b, h) of out at
+ * out + b * out_stride_seq + h * D: the H heads of one sequence stay contiguous, consecutive
+ * sequences are q_stride_seq / out_stride_seq elements apart (each >= H * D and a multiple of
+ * 8, else PA_ERR_ARG / PA_ERR_ALIGN).  Everything else, errors included, is pa_decode's; with
+ * both strides equal to H * D the two calls are the same.  The cache slice of a rank is described
+ * by `shape` as always (its strides may be those of a wider pool).
+ */
+int pa_decode_strided(const pa_shape* shape, const void* q, int64_t q_stride_seq,
+                      const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                      int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
+                      float scale, void* out, int64_t out_stride_seq, void* workspace,
+                      size_t workspace_bytes, int32_t partition_tokens, int32_t flags,
+                      int32_t* dev_status, void* cuda_stream);
 
 /*
  * pa_decode for callers that cannot allocate device memory.  (The paper has no counterpart;

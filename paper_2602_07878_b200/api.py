@@ -27,7 +27,7 @@ ERR = {"NULL": -1, "SHAPE": -2, "ALIGN": -3, "WORKSPACE": -4, "HOSTBUF": -5, "BL
        "CUDA": -7, "ARG": -8, "STATIC_LIMIT": -9}
 PA_STATIC_WORKSPACE_BYTES = 64 << 20
 
-EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_host_io_bytes", "pa_decode_host",
+EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_decode_strided", "pa_host_io_bytes", "pa_decode_host",
            "kv_block_bytes", "kv_swap_out", "kv_swap_in", "pa_status_string",
            "pa_last_cuda_error", "pa_launch_count", "pa_profile_enable", "pa_profile_read",
            "pa_decode_static", "kv_append", "pa_partial_floats", "pa_decode_partial",
@@ -105,6 +105,9 @@ def lib() -> ctypes.CDLL:
         L.pa_probe_read.restype = ctypes.c_int
         L.kv_append.argtypes = [pshape, vp, vp, vp, vp, vp, i32, vp, vp]
         L.kv_append.restype = ctypes.c_int
+        L.pa_decode_strided.argtypes = [pshape, vp, ctypes.c_int64, vp, vp, vp, i32, vp, i32,
+                                        ctypes.c_float, vp, ctypes.c_int64, vp, sz, i32, i32, vp, vp]
+        L.pa_decode_strided.restype = ctypes.c_int
         L.pa_host_io_bytes.argtypes = [pshape, i32, i32, psz]
         L.pa_decode_host.argtypes = [pshape, vp, vp, vp, vp, i32, vp, i32, ctypes.c_float, vp, vp,
                                      sz, vp, sz, i32, vp, vp]
@@ -168,13 +171,26 @@ def pa_decode(q, k_cache, v_cache, block_tables, seq_lens, scale, out, workspace
         shape = shape_of(k_cache, q.shape[1])
         assert v_cache.stride() == k_cache.stride() and v_cache.shape == k_cache.shape
     assert block_tables.dtype == torch.int32 and seq_lens.dtype == torch.int32
-    assert q.is_contiguous() and out.is_contiguous() and block_tables.is_contiguous()
-    rc = lib().pa_decode(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
-                         _ptr(block_tables), block_tables.shape[1] if block_tables.dim() == 2 else 0,
-                         _ptr(seq_lens), q.shape[0], float(scale), _ptr(out), _ptr(workspace),
-                         workspace.numel() * workspace.element_size(), partition_tokens, flags,
-                         _ptr(dev_status), _stream(stream))
-    _check(rc, "pa_decode")
+    assert block_tables.is_contiguous()
+    max_blocks = block_tables.shape[1] if block_tables.dim() == 2 else 0
+    if q.is_contiguous() and out.is_contiguous():
+        rc = lib().pa_decode(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                             _ptr(block_tables), max_blocks, _ptr(seq_lens), q.shape[0],
+                             float(scale), _ptr(out), _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), partition_tokens, flags,
+                             _ptr(dev_status), _stream(stream))
+        _check(rc, "pa_decode")
+        return out
+    # views into wider tensors (a rank's heads of a batch-wide q, the q part of a fused QKV
+    # projection): each sequence's [H, D] rows must be contiguous, sequences may be further apart
+    for t in (q, out):
+        assert t.dim() == 3 and t.stride(2) == 1 and t.stride(1) == t.shape[2]
+    rc = lib().pa_decode_strided(ctypes.byref(shape), _ptr(q), q.stride(0), _ptr(k_cache),
+                                 _ptr(v_cache), _ptr(block_tables), max_blocks, _ptr(seq_lens),
+                                 q.shape[0], float(scale), _ptr(out), out.stride(0),
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                 partition_tokens, flags, _ptr(dev_status), _stream(stream))
+    _check(rc, "pa_decode_strided")
     return out
 
 

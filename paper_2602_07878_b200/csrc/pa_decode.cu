@@ -224,6 +224,9 @@ struct DecodeParams {
     int* status;
     int max_blocks, H, Hkv, G, NB;
     float scale_log2;
+    // elements between the [H, D] rows of consecutive sequences in q and in out (H * D when
+    // they are contiguous; larger when they are views into wider tensors)
+    int64_t q_stride, out_stride;
 };
 
 
@@ -306,7 +309,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         u.id = 0;
         if (valid && lane < u.nblk)
             u.id = __ldg(&p.block_tables[(size_t)u.b * p.max_blocks + u.tok0 / BS + lane]);
-        const size_t row0 = valid ? ((size_t)u.b * H + (size_t)kvh * G) * D : 0;
+        const size_t row0 = valid ? (size_t)u.b * p.q_stride + (size_t)kvh * G * D : 0;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
             // a0: (row g, k 2t..), a2: (row g, k 8+2t..); a1/a3 the same for row g+8
@@ -413,14 +416,15 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             if (U0.direct) {
                 const float i0 = U0.bad ? 0.f : 1.f / l0, i1 = U0.bad ? 0.f : 1.f / l1;
                 if (g < G) {
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(p.out + ((size_t)U0.b * H + h0) * D);
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(
+                        p.out + (size_t)U0.b * p.out_stride + (size_t)h0 * D);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
                         dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0);
                 }
                 if (HI && g + 8 < G) {
-                    uint32_t* dst =
-                        reinterpret_cast<uint32_t*>(p.out + ((size_t)U0.b * H + h0 + 8) * D);
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(
+                        p.out + (size_t)U0.b * p.out_stride + (size_t)(h0 + 8) * D);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
                         dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][2] * i1, o[nt][3] * i1);
@@ -468,6 +472,7 @@ struct CombineParams {
     int* hdr;
     int rows;  // batch * H
     int H;
+    int64_t out_stride;  // elements between the [H, D] output rows of consecutive sequences
     int counter_reset;
     // COMBINE_TO_PARTIAL: one un-normalised fp32 row and its (max, sum) per output row
     float* part_o;
@@ -496,7 +501,7 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const __grid_constant__
     const int b = row / p.H, h = row - b * p.H;
     const int2 info = MODE == COMBINE_MERGE ? make_int2(0, p.n_parts) : p.seq_info[b];
     if (MODE == COMBINE_FINAL && info.y == 1) return;  // written directly by the attention kernel
-    __nv_bfloat16* dst = p.out + (size_t)row * D;
+    __nv_bfloat16* dst = p.out + (size_t)b * p.out_stride + (size_t)h * D;
     if (info.y == 0) {  // no tokens: a row of zeros (as a partial: weight zero)
         if (MODE == COMBINE_TO_PARTIAL) {
             if (threadIdx.x < D / 2)
@@ -914,7 +919,7 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
                 for (int w = 0; w < 8; ++w) t += s_acc[w][lane * VPL + i];
                 o[i] = t * inv;
             }
-            store(p.out + ((size_t)b * p.H + h) * D + lane * VPL, o, zero);
+            store(p.out + (size_t)b * p.out_stride + (size_t)h * D + lane * VPL, o, zero);
         }
         __syncthreads();
     }
@@ -934,7 +939,7 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
         const float inv = zero ? 0.f : 1.f / den;
 #pragma unroll
         for (int i = 0; i < VPL; ++i) acc[i] *= inv;
-        store(p.out + ((size_t)b * p.H + h) * D + lane * VPL, acc, zero);
+        store(p.out + (size_t)b * p.out_stride + (size_t)h * D + lane * VPL, acc, zero);
     }
 }
 
@@ -952,7 +957,8 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
                        int32_t max_blocks_per_seq, const int32_t* seq_lens, int32_t batch,
                        float scale, void* out, float* part, void* workspace,
                        size_t workspace_bytes, int32_t partition_tokens, int32_t flags,
-                       int32_t* dev_status, void* cuda_stream) {
+                       int32_t* dev_status, void* cuda_stream, int64_t q_stride = 0,
+                       int64_t out_stride = 0) {
     if (!shape) return PA_ERR_NULL;
     int rc = validate_shape(shape);
     if (rc) return rc;
@@ -971,6 +977,12 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     if ((int64_t)max_blocks_per_seq * BS > INT32_MAX) return PA_ERR_ARG;
 
     const int H = shape->num_q_heads, D = shape->head_dim;
+    // 0 = contiguous; otherwise at least one [H, D] row apart and a multiple of 8 elements so
+    // that every row stays 16-byte aligned
+    if (q_stride == 0) q_stride = (int64_t)H * D;
+    if (out_stride == 0) out_stride = (int64_t)H * D;
+    if (q_stride < (int64_t)H * D || out_stride < (int64_t)H * D) return PA_ERR_ARG;
+    if ((q_stride | out_stride) & 7) return PA_ERR_ALIGN;
     WsLayout w = ws_layout(H, D, batch, 0, workspace_bytes);
     if (w.item_cap < batch || w.total > workspace_bytes) return PA_ERR_WORKSPACE;
 
@@ -1003,6 +1015,8 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     dp.G = H / shape->num_kv_heads;
     dp.NB = shape->num_blocks;
     dp.scale_log2 = scale * 1.4426950408889634f;
+    dp.q_stride = q_stride;
+    dp.out_stride = out_stride;
 
     int total_warps = 0;
     rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, false, st);
@@ -1045,6 +1059,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     cp.hdr = hdr;
     cp.rows = batch * H;
     cp.H = H;
+    cp.out_stride = out_stride;
     cp.counter_reset = 3 * total_warps;
     if (part) {
         cp.part_o = part;
@@ -1070,6 +1085,19 @@ extern "C" int pa_decode(const pa_shape* shape, const void* q, const void* k_cac
     return decode_impl(shape, q, k_cache, v_cache, block_tables, max_blocks_per_seq, seq_lens,
                        batch, scale, out, nullptr, workspace, workspace_bytes, partition_tokens,
                        flags, dev_status, cuda_stream);
+}
+
+extern "C" int pa_decode_strided(const pa_shape* shape, const void* q, int64_t q_stride_seq,
+                                 const void* k_cache, const void* v_cache,
+                                 const int32_t* block_tables, int32_t max_blocks_per_seq,
+                                 const int32_t* seq_lens, int32_t batch, float scale, void* out,
+                                 int64_t out_stride_seq, void* workspace, size_t workspace_bytes,
+                                 int32_t partition_tokens, int32_t flags, int32_t* dev_status,
+                                 void* cuda_stream) {
+    if (q_stride_seq <= 0 || out_stride_seq <= 0) return PA_ERR_ARG;
+    return decode_impl(shape, q, k_cache, v_cache, block_tables, max_blocks_per_seq, seq_lens,
+                       batch, scale, out, nullptr, workspace, workspace_bytes, partition_tokens,
+                       flags, dev_status, cuda_stream, q_stride_seq, out_stride_seq);
 }
 
 extern "C" int pa_partial_floats(const pa_shape* shape, int32_t batch, size_t* floats) {
@@ -1110,6 +1138,7 @@ extern "C" int pa_merge_partials(const float* const* parts, int32_t num_parts, i
     cp.out = static_cast<__nv_bfloat16*>(out);
     cp.rows = rows;
     cp.H = 1;
+    cp.out_stride = head_dim;
     cp.n_parts = num_parts;
     DeviceInfo dev;
     int rc = get_device_info(&dev);
