@@ -173,7 +173,10 @@ int pa_decode_strided(const pa_shape* shape, const void* q, int64_t q_stride_seq
  * are still the caller's.
  *
  * First call on each device: the array's device address is looked up once per device (with
- * that device current) and cached.  Make that first call outside any stream capture.
+ * that device current) and cached.  Make that first call outside any stream capture.  On every
+ * call the device that owns `cuda_stream` must be the current device (the cached address is
+ * chosen by the current device's ordinal), and the cache does not survive cudaDeviceReset: a
+ * process that resets a device must not call this entry point on it afterwards.
  * Sharing: all calls on a device use the same array, and it keeps what the last call left
  * there.  The call clears the plan header before use; everything else is overwritten
  * before it is read.  Two calls whose GPU work overlaps (different streams, or different

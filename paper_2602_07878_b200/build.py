@@ -11,7 +11,7 @@ LIB = os.path.join(_HERE, "libpagedkv.so")
 SOURCES = ["common.cu", "pa_decode.cu", "kv_swap.cu", "kv_append.cu", "pa_prefill.cu", "probes.cu", "sched_sim.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math", "-Xcompiler", "-fPIC", "-Xptxas", "-v", "--threads", "0",
+    "-Xcompiler", "-fPIC", "-Xptxas", "-v", "--threads", "0",
 ]
 
 

@@ -5,6 +5,8 @@
 // bulk asynchronous copy into shared memory per granule, completion counted on an mbarrier.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -96,12 +98,18 @@ extern "C" int pa_probe_read(const void* dev_buf, size_t bytes, int32_t scattere
     int rc = get_device_info(&dev);
     if (rc) return rc;
     const int smem = PROBE_WARPS * PROBE_SLOTS * PROBE_GRANULE + PROBE_WARPS * PROBE_SLOTS * 8 + 128;
-    static int configured_dev = -1;
-    if (configured_dev != dev.device) {
-        rc = check_cuda(cudaFuncSetAttribute(probe_read_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        if (rc) return rc;
-        configured_dev = dev.device;
+    // the attribute is set once per device; callers may come from several host threads
+    static std::mutex mu;
+    static bool configured[64] = {false};
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (dev.device < 0 || dev.device >= 64) return PA_ERR_ARG;
+        if (!configured[dev.device]) {
+            rc = check_cuda(cudaFuncSetAttribute(
+                probe_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            if (rc) return rc;
+            configured[dev.device] = true;
+        }
     }
     probe_read_kernel<<<dev.sm_count, PROBE_WARPS * 32, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
         static_cast<const uint8_t*>(dev_buf), (unsigned long long)(bytes / PROBE_GRANULE),
