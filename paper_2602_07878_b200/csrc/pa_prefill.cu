@@ -321,7 +321,12 @@ struct Cfg {
     static constexpr int TMEM_COLS = NT * TILE_COLS <= 256 ? 256 : 512;
     static_assert(NT * TILE_COLS <= 512, "tensor memory holds 512 columns");
     static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
-    static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + 1, THREADS = (4 * NT + 2) * 32;
+    // Four TMA producer warps, one per 16-token block of a step: a warp pays some 400 cycles
+    // per bulk-tensor instruction plus about 45 per lane that issues a box in it, so one warp
+    // issuing the 16 boxes (2 KB each) of a head_dim-128 step cannot keep up with the MMAs.
+    static constexpr int N_PRODUCERS = 4;
+    static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + N_PRODUCERS,
+                         THREADS = (4 * NT + N_PRODUCERS + 1) * 32;
 };
 // per-tile barrier indices, relative to Cfg::B_TILE + 8 * tile
 enum { T_SFULL = 0, T_PFULL = 2, T_PVDONE = 4 };
@@ -423,8 +428,11 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
-        for (int i = 0; i < KS; ++i) mbar_init(bar(B_KFULL + i), 1), mbar_init(bar(B_KEMPTY + i), 1);
-        for (int i = 0; i < VS; ++i) mbar_init(bar(B_VFULL + i), 1), mbar_init(bar(B_VEMPTY + i), 1);
+        // a K/V stage is full once each producer warp has announced and delivered its block
+        for (int i = 0; i < KS; ++i)
+            mbar_init(bar(B_KFULL + i), C::N_PRODUCERS), mbar_init(bar(B_KEMPTY + i), 1);
+        for (int i = 0; i < VS; ++i)
+            mbar_init(bar(B_VFULL + i), C::N_PRODUCERS), mbar_init(bar(B_VEMPTY + i), 1);
         for (int t = 0; t < NT; ++t)
             for (int i = 0; i < 2; ++i) {
                 mbar_init(bar(C::B_TILE + 8 * t + T_SFULL + i), 1);
@@ -463,35 +471,43 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         return false;
     };
 
-    if (warp == C::PRODUCER_WARP) {
-        // ===================== TMA producer =====================
-        if (lane == 0) {
+    if (warp >= C::PRODUCER_WARP && warp < C::PRODUCER_WARP + C::N_PRODUCERS) {
+        // ===================== TMA producers =====================
+        // Warp pw fetches block pw of every 64-token step: its K boxes and its V boxes, one box
+        // (64 dims x 16 tokens) per lane.
+        const int pw = warp - C::PRODUCER_WARP;
+        if (pw == 0 && lane == 0) {
             tma_prefetch_desc(&qmap);
-            tma_prefetch_desc(&kmap);
-            tma_prefetch_desc(&vmap);
             mbar_arrive_expect_tx(bar(B_QFULL), NT * NG * rows_used * 128);
             for (int t = 0; t < NT; ++t)  // tile t holds query tokens tok0 + t * tpt ..
                 for (int g = 0; g < NG; ++g)
                     tma_load_4d(sbase + OFF_Q + t * Q_BYTES + g * C::Q_GROUP, &qmap, bar(B_QFULL),
                                 g * 64, 0, kvh, q0 + tok0 + t * tpt);
         }
+        if (lane == 0) {
+            tma_prefetch_desc(&kmap);
+            tma_prefetch_desc(&vmap);
+        }
         const int32_t* table = p.block_tables + (size_t)b * p.max_blocks;
         // block ids are fetched 32 at a time, one window ahead; the unit starts at block 4 * j0
         const int win0 = (j0 * 4) & ~31;
         int ids = win0 + lane < nblk_seq ? __ldg(&table[win0 + lane]) : p.NB;
         int ids_next = win0 + 32 + lane < nblk_seq ? __ldg(&table[win0 + 32 + lane]) : p.NB;
-        // lane l < 4 * NG: block l / NG of the step, column group l % NG
-        const int blk = lane / NG, grp = lane - blk * NG;
-        const uint32_t tile_off = grp * GROUP_BYTES + blk * (BS * 128);
+        // shared rings: lanes [0, NG) take the K boxes, [NG, 2 NG) the V boxes, one instruction;
+        // split rings: lanes [0, NG) issue K, then V, each against its own barrier
+        const bool is_v = !SPLIT && lane >= NG;
+        const int grp = is_v ? lane - NG : lane;
+        const uint32_t tile_off = grp * GROUP_BYTES + pw * (BS * 128);
+        constexpr uint32_t BLOCK_BYTES = TILE_BYTES / 4;  // K (or V) of one block, all column groups
         for (int j = 0; j < n_steps; ++j) {
             const int blk0 = (j0 + j) * 4;
             if (blk0 > win0 && (blk0 & 31) == 0) {
                 ids = ids_next;
                 ids_next = blk0 + 32 + lane < nblk_seq ? __ldg(&table[blk0 + 32 + lane]) : p.NB;
             }
-            const int id = __shfl_sync(0xffffffffu, ids, (blk0 + (blk & 3)) & 31);
-            const bool used = blk0 + blk < nblk_seq;
-            if (lane < 4 * NG && used && (unsigned)id >= (unsigned)p.NB && grp == 0) {
+            const int id = __shfl_sync(0xffffffffu, ids, (blk0 + pw) & 31);
+            const bool used = blk0 + pw < nblk_seq;
+            if (lane == 0 && used && (unsigned)id >= (unsigned)p.NB) {
                 misc[2] = 1;
                 atomicOr(p.status, PA_STATUS_BAD_BLOCK_ID);
             }
@@ -500,23 +516,25 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
             const int ks = j % KS, vs = j % VS;
             if (SPLIT) {
                 if (j >= KS && !wait(B_KEMPTY + ks, ((j / KS) - 1) & 1)) break;
-                if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), TILE_BYTES);
+                if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), BLOCK_BYTES);
+                __syncwarp();
+                if (lane < NG)
+                    tma_load_4d(sbase + OFF_K + ks * TILE_BYTES + tile_off, &kmap, bar(B_KFULL + ks),
+                                grp * 64, 0, kvh, coord);
+                if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
+                if (lane == 0) mbar_arrive_expect_tx(bar(B_VFULL + vs), BLOCK_BYTES);
+                __syncwarp();
+                if (lane < NG)
+                    tma_load_4d(sbase + OFF_V + vs * TILE_BYTES + tile_off, &vmap, bar(B_VFULL + vs),
+                                grp * 64, 0, kvh, coord);
             } else {
                 if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
-                if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), 2 * TILE_BYTES);
-            }
-            __syncwarp();
-            if (lane < 4 * NG)
-                tma_load_4d(sbase + OFF_K + ks * TILE_BYTES + tile_off, &kmap, bar(B_KFULL + ks),
-                            grp * 64, 0, kvh, coord);
-            if (SPLIT) {
-                if (j >= VS && !wait(B_VEMPTY + vs, ((j / VS) - 1) & 1)) break;
-                if (lane == 0) mbar_arrive_expect_tx(bar(B_VFULL + vs), TILE_BYTES);
+                if (lane == 0) mbar_arrive_expect_tx(bar(B_KFULL + ks), 2 * BLOCK_BYTES);
                 __syncwarp();
+                if (lane < 2 * NG)
+                    tma_load_4d(sbase + (is_v ? OFF_V + vs * TILE_BYTES : OFF_K + ks * TILE_BYTES) + tile_off,
+                                is_v ? &vmap : &kmap, bar(B_KFULL + ks), grp * 64, 0, kvh, coord);
             }
-            if (lane < 4 * NG)
-                tma_load_4d(sbase + OFF_V + vs * TILE_BYTES + tile_off, &vmap, bar(B_VFULL + vs),
-                            grp * 64, 0, kvh, coord);
         }
     } else if (warp == C::MMA_WARP) {
         // ===================== MMA issuer =====================
