@@ -415,9 +415,13 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     const int b = lo;
     const int q0 = p.cu_q_lens[b], ql = p.cu_q_lens[b + 1] - q0, L = p.ctx_lens[b];
     const int n_split = kv_splits(L, tp.split_steps);   // units per row group of this sequence
+    // Units of a sequence in launch order (blockIdx ascending = u descending): split 0 of every
+    // row group, later row groups first, then split 1, ...  The last split is the short one
+    // when the split length does not divide the context, and short units fill the SMs last.
     const int r = gi - gs[b];
-    const int split = r % n_split;
-    const int tok0 = (r / n_split) * (NT * tpt);        // first query token of the CTA
+    const int n_groups_b = (ql + p.tpg - 1) / p.tpg;    // row groups (CTAs per split) of this sequence
+    const int split = n_split - 1 - r / n_groups_b;
+    const int tok0 = (r % n_groups_b) * (NT * tpt);     // first query token of the CTA
     const int ntok_cta = min(NT * tpt, ql - tok0);
     const int pos_max = L - ql + tok0 + ntok_cta - 1;
     const int j0 = split * tp.split_steps;              // first 64-token step of this unit
@@ -1016,6 +1020,18 @@ namespace pk {
 struct TcShape {
     int tiles_per_cta, split_steps, split_cap;
 };
+// Time of `n_long` units of cost `cl` and `n_short` units of cost `cs` <= cl on `M` SMs when
+// the long ones start first and every SM takes the next unit as it becomes free.
+static double makespan(int64_t n_long, double cl, int64_t n_short, double cs, int M) {
+    const int64_t a = n_long / M, e = n_long % M;
+    if (n_short == 0) return (double)(a + (e > 0)) * cl;
+    if (e == 0) return a * cl + (double)((n_short + M - 1) / M) * cs;
+    // M - e SMs are one long unit behind the others and take short ones until they catch up
+    const int64_t k = std::max<int64_t>(1, (int64_t)(cl / cs)), cap = (M - e) * k;
+    if (n_short <= cap) return (a + 1) * cl;
+    return (a + 1) * cl + (double)((n_short - cap + M - 1) / M) * cs;
+}
+
 static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H, int D,
                                int64_t steps_bound, int sm_count, int64_t cap_fit,
                                int forced_tiles, int forced_split_steps) {
@@ -1029,20 +1045,33 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
             (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
         // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
         // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
-        const double step_us = D == 256 ? 1.40 : D == 64 ? (nt == 1 ? 0.66 : 0.88) : (nt == 1 ? 0.83 : 0.92);
-        const int64_t s_hi = forced_split_steps ? 1 : std::min<int64_t>({cap_fit, 64, steps_bound / 8});
-        for (int64_t s_try = 1; s_try <= std::max<int64_t>(1, s_hi); ++s_try) {
-            int64_t T = forced_split_steps ? forced_split_steps : (steps_bound + s_try - 1) / s_try;
+        const double step_us = D == 256 ? 1.10 : D == 64 ? (nt == 1 ? 0.66 : 0.88) : (nt == 1 ? 0.80 : 0.86);
+        const double unit_us = 8.0;
+        auto consider = [&](int64_t T) {
+            T = std::min(std::max<int64_t>(T, 1), steps_bound);
             const int64_t S = (steps_bound + T - 1) / T;
-            if (S > cap_fit && S > 1) continue;
-            const int64_t rounds = (groups * S + sm_count - 1) / sm_count;
-            double t = rounds * (T * step_us + 10.0);
+            if (S > 1 && (S > cap_fit || (S > 64 && !forced_split_steps))) return;
+            if (S > 1 && !forced_split_steps && T < 8) return;  // a unit must be worth its set-up
+            const int64_t r = steps_bound - (S - 1) * T;        // steps of the last split
+            const bool even = r == T;
+            double t = makespan(even ? groups * S : groups * (S - 1), T * step_us + unit_us,
+                                even ? 0 : groups, r * step_us + unit_us, sm_count);
             if (S > 1) t += 6.0 + (double)total_q * H * S * (D + 2) * 4 * 2 / 5.0e6;
             if (t < best_t) {
                 best_t = t;
                 best = {nt, S > 1 ? (int)T : 0, (int)std::max<int64_t>(S, 1)};
             }
+        };
+        if (forced_split_steps) {
+            consider(forced_split_steps);
+            continue;
         }
+        // even splits, and split lengths in between (a short last split fills SMs that a
+        // whole number of equal units would leave idle)
+        for (int64_t S = 1; S <= std::max<int64_t>(1, std::min<int64_t>(cap_fit, 64)); ++S)
+            consider((steps_bound + S - 1) / S);
+        if (cap_fit > 1)
+            for (int64_t i = 1; i < 48; ++i) consider(steps_bound * i / 48);
     }
     return best;
 }

@@ -24,8 +24,14 @@ def test_recompute_chunk_of_one_long_sequence_is_split_over_the_sms():
     tiles, tok, splits = api.pa_prefill_select_launch(sh, 1, 512, 2048, ws(sh, 1, 512, 16))
     assert tiles == 2 and splits >= 2 and tok % 64 == 0
     assert tok * splits >= 32768 > tok * (splits - 1)         # the splits cover the context
-    units = 512 // (2 * 32) * 8 * splits
-    assert units <= 148 or units >= 2 * 148 - 148 // 4       # one full round, or several
+    # 64 row groups x splits: the full-length units fill one round of the 148 SMs and the
+    # shorter last split of every row group fits on the SMs they leave free
+    groups = 512 // (2 * 32) * 8
+    n_long, last = groups * (splits - 1), 32768 - tok * (splits - 1)
+    assert n_long <= 148 and 0 < last <= tok
+    if last < tok:
+        per_free_sm = -(-groups // (148 - n_long))
+        assert per_free_sm * last <= tok
 
 
 def test_no_split_without_room_for_partial_rows_or_on_request():
