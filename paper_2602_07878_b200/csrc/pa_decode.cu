@@ -66,6 +66,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     __shared__ int hist[MAX_PART / BS + 1], start[MAX_PART / BS + 1], cursor[MAX_PART / BS + 1];
     __shared__ int scan_warp[32];
     __shared__ int s_carry, s_multi, s_long;
+    // (length, first partial index) of the first PLAN_THREADS sequences: pass 3 reads them here
+    // instead of loading back what pass 2 has just written to global memory
+    __shared__ int2 s_seq[PLAN_THREADS];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int max_tok = p.max_blocks * BS;
@@ -92,11 +95,14 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     if (tid < MAX_PART / BS + 1) hist[tid] = 0, cursor[tid] = 0;
     __syncthreads();
     if (bad) s_bad = 1;
-    if (tid == 0) {
+    if (warp == 0) {
+        // lane w holds warp w's counts; one shuffle tree per candidate, every lane ends with
+        // the totals
         long long tot[5];
+#pragma unroll
         for (int c = 0; c < 5; ++c) {
-            long long v = 0;
-            for (int w = 0; w < PLAN_THREADS / 32; ++w) v += red[c][w];
+            long long v = red[c][lane];
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
             tot[c] = v;
         }
         int P = 0;
@@ -112,8 +118,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
                 if (tot[c] * p.Hkv >= want) break;
             }
         }
-        s_P = P;
-        s_carry = 0;
+        if (lane == 0) {
+            s_P = P;
+            s_carry = 0;
+        }
     }
     __syncthreads();
     const int P = s_P;
@@ -170,18 +178,31 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
         __syncthreads();
         const int warp_off = warp == 0 ? 0 : scan_warp[warp - 1];
         const int carry = s_carry;
-        if (b < p.batch) p.seq_info[b] = make_int2(carry + warp_off + incl - np, np);
+        if (b < p.batch) {
+            const int first = carry + warp_off + incl - np;
+            p.seq_info[b] = make_int2(first, np);
+            if (base == 0) {
+                bool dummy = false;
+                s_seq[tid] = make_int2(clamp_len(p.seq_lens[b], max_tok, dummy), first);
+            }
+        }
         __syncthreads();
         if (tid == 0) s_carry = carry + scan_warp[31];
         __syncthreads();
     }
     const int n_items = s_carry;
-    if (tid == 0) {
-        int acc = 0;  // larger items first
-        for (int nb = MAX_PART / BS; nb >= 1; --nb) {
-            start[nb] = acc;
-            acc += hist[nb];
+    if (warp == 0) {  // larger items first: exclusive scan of the histogram from the top bin down
+        static_assert(MAX_PART / BS == 32, "one lane per bin");
+        const int nb = MAX_PART / BS - lane;
+        const int v = hist[nb];
+        int incl = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += u;
         }
+        start[nb] = incl - v;
+    }
+    if (tid == 0) {
         p.hdr[HDR_N_ITEMS] = n_items;
         p.hdr[HDR_N_MULTI] = s_multi;
         p.hdr[HDR_N_LONG] = s_long;
@@ -195,10 +216,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     // ---- pass 3: one warp per sequence, lanes over its partitions ------------------------
     for (int b = warp; b < p.batch; b += PLAN_THREADS / 32) {
         bool dummy = false;
-        const int L = clamp_len(p.seq_lens[b], max_tok, dummy);
+        const int L = b < PLAN_THREADS ? s_seq[b].x : clamp_len(p.seq_lens[b], max_tok, dummy);
         const int np = (L + P - 1) / P;
         if (np == 0) continue;
-        const int first = p.seq_info[b].x;
+        const int first = b < PLAN_THREADS ? s_seq[b].y : p.seq_info[b].x;
         for (int part = lane; part < np; part += 32) {
             const int tok0 = part * P;
             const int ntok = min(P, L - tok0);
@@ -272,8 +293,11 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         tma_prefetch_desc(&vmap);
     }
     __syncwarp();
-    pdl_launch_dependents();  // combine CTAs may take their seats; they wait for this grid
     pdl_wait();               // the plan (and everything before it) is complete and visible
+    // Only now may the combine CTAs take their seats: they start once every CTA of this grid
+    // has passed this point, i.e. after the plan grid has completed, so the plan's lists are
+    // theirs to read even before they wait for this grid's partial results.
+    pdl_launch_dependents();
 
     const int n_units = p.hdr[HDR_N_UNITS];
     const int total_warps = NW * gridDim.x;
@@ -827,9 +851,23 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
     __shared__ float s_den[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     pdl_launch_dependents();
+    // The plan's lists were complete before this grid could start (the attention kernel lets
+    // its dependents go only after it has seen the plan), so the chain header -> list entry ->
+    // sequence record of this CTA's first rows is walked while the attention kernel still runs.
+    const int batch = p.rows / p.H;
+    const int n_long = p.hdr[HDR_N_LONG] * p.H, n_short = p.hdr[HDR_N_MULTI] * p.H;
+    int2 first_long = make_int2(0, 0), first_short = make_int2(0, 0);
+    int first_long_b = 0, first_short_b = 0;
+    if ((int)blockIdx.x < n_long) {
+        first_long_b = __ldg(&p.multi[blockIdx.x / p.H]);
+        first_long = p.seq_info[first_long_b];
+    }
+    if ((int)blockIdx.x * 8 + warp < n_short) {
+        first_short_b = __ldg(&p.multi[batch - 1 - (blockIdx.x * 8 + warp) / p.H]);
+        first_short = p.seq_info[first_short_b];
+    }
     pdl_wait();  // partial results of the attention kernel are complete and visible
     if (blockIdx.x == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
-    const int n_long = p.hdr[HDR_N_LONG] * p.H, n_short = p.hdr[HDR_N_MULTI] * p.H;
 
     // sum of w_i * (o_i, l_i) over partitions i = start, start + stride, ... < np of one row
     auto gather = [&](int first, int np, int h, int start, int stride, float M, float (&acc)[VPL],
@@ -892,8 +930,9 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
 
     // ---- long rows: one per CTA ----
     for (int task = blockIdx.x; task < n_long; task += gridDim.x) {
-        const int b = __ldg(&p.multi[task / p.H]), h = task % p.H;
-        const int2 info = p.seq_info[b];
+        const bool first = task == (int)blockIdx.x;
+        const int b = first ? first_long_b : __ldg(&p.multi[task / p.H]), h = task % p.H;
+        const int2 info = first ? first_long : p.seq_info[b];
         bool bad;
         const float M = row_max(info.x, info.y, h, bad);
         float acc[VPL];
@@ -924,10 +963,10 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
         __syncthreads();
     }
     // ---- short rows: one per warp ----
-    const int batch = p.rows / p.H;
     for (int task = blockIdx.x * 8 + warp; task < n_short; task += gridDim.x * 8) {
-        const int b = __ldg(&p.multi[batch - 1 - task / p.H]), h = task % p.H;
-        const int2 info = p.seq_info[b];
+        const bool first = task == (int)blockIdx.x * 8 + warp;
+        const int b = first ? first_short_b : __ldg(&p.multi[batch - 1 - task / p.H]), h = task % p.H;
+        const int2 info = first ? first_short : p.seq_info[b];
         bool bad;
         const float M = row_max(info.x, info.y, h, bad);
         float acc[VPL];
