@@ -371,8 +371,11 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + OFF_MISC);
     // misc[0] = TMEM base address, misc[1] = abort flag, misc[2] = bad block id seen
 
-    pdl_launch_dependents();
+    // Dependents (the merge kernel, the next call) start once every CTA here has passed the
+    // wait, i.e. when all that precedes this call in the stream is complete: they may then read
+    // the call's inputs before they wait for this grid themselves.
     pdl_wait();
+    pdl_launch_dependents();
 
     // ---- which tile -------------------------------------------------------------------------
     const int G = p.G, H = p.H, Hkv = p.Hkv, tpt = tp.tokens_per_tile;
@@ -840,28 +843,35 @@ template <int D>
 __global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMergeParams p) {
     constexpr int NV = (D / 4 + 31) / 32;  // float4 pieces of a row per lane
     pdl_launch_dependents();
-    pdl_wait();
+    // the lengths are inputs of the call, complete before the attention kernel let this grid
+    // start: the row's sequence and its number of splits are worked out while attention runs
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (row >= (long long)p.total_q * p.H) return;
-    const int qi = (int)(row / p.H);
-    int lo = 0, hi = p.batch;  // last b with cu_q_lens[b] <= qi
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (__ldg(&p.cu_q_lens[mid]) <= qi) lo = mid; else hi = mid;
+    int n_vis = 0;  // stays 0 for a row this kernel leaves alone
+    if (row < (long long)p.total_q * p.H) {
+        const int qi = (int)(row / p.H);
+        int lo = 0, hi = p.batch;  // last b with cu_q_lens[b] <= qi
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (__ldg(&p.cu_q_lens[mid]) <= qi) lo = mid; else hi = mid;
+        }
+        const int b = lo;
+        const int q0 = __ldg(&p.cu_q_lens[b]), q1 = __ldg(&p.cu_q_lens[b + 1]), L = __ldg(&p.ctx_lens[b]);
+        const int ql = q1 - q0;
+        const bool ok = q0 >= 0 && ql >= 0 && q1 <= p.total_q && L >= ql &&
+                        L <= p.max_blocks * BS && (b > 0 || q0 == 0) && qi >= q0 && qi < q1;
+        const int n_split = ok ? kv_splits(L, p.split_steps) : 1;
+        if (n_split > 1) {
+            // splits visited by the row's tile group: those that start at or before its last position
+            const int tok0 = (qi - q0) / p.tpg * p.tpg;
+            const int pos_max = L - ql + min(tok0 + p.tpg, ql) - 1;
+            n_vis = min(n_split, (pos_max / 64 + 1 + p.split_steps - 1) / p.split_steps);
+        }
     }
-    const int b = lo;
-    const int q0 = __ldg(&p.cu_q_lens[b]), q1 = __ldg(&p.cu_q_lens[b + 1]), L = __ldg(&p.ctx_lens[b]);
-    const int ql = q1 - q0;
-    const bool ok = q0 >= 0 && ql >= 0 && q1 <= p.total_q && L >= ql &&
-                    L <= p.max_blocks * BS && (b > 0 || q0 == 0) && qi >= q0 && qi < q1;
-    if (!ok) return;
-    const int n_split = kv_splits(L, p.split_steps);
-    if (n_split <= 1) return;
-    // splits visited by the row's tile group: those that start at or before its last position
-    const int tok0 = (qi - q0) / p.tpg * p.tpg;
-    const int pos_max = L - ql + min(tok0 + p.tpg, ql) - 1;
-    const int n_vis = min(n_split, (pos_max / 64 + 1 + p.split_steps - 1) / p.split_steps);
+    // every thread waits before it leaves: the grid must not count as complete, and let the
+    // next kernel in the stream go, before the attention kernel has finished
+    pdl_wait();
+    if (n_vis == 0) return;
     const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + (size_t)row * p.split_cap;
     float M = -INFINITY;
     bool bad = false;
