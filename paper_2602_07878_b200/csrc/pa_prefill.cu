@@ -288,10 +288,15 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 // buffers and a ring of K/V tiles let Q K^T of step j+1 overlap the softmax of step j.
 namespace tc {
 constexpr int ROWS = 128, STEP = 64;
+// Of every 8 pairs of weights, how many take the packed cubic on the FMA pipe instead of EX2.
+// With one TMA producer warp the special-function unit was the scarcer resource and 2 was
+// best; since the K/V feed keeps up, the softmax warps are bound by instruction issue and the
+// cubic's extra instructions cost more than they save (512-token recompute leg: 1110 TFLOP/s
+// at 0, 1103 at 1, 1083 at 2, 1057 at 3, 1012 at 4).
 #ifndef PAGEDKV_POLY_PAIRS
-#define PAGEDKV_POLY_PAIRS 2
+#define PAGEDKV_POLY_PAIRS 0
 #endif
-constexpr int POLY_PAIRS = PAGEDKV_POLY_PAIRS;  // of every 8 pairs of weights, how many take the cubic
+constexpr int POLY_PAIRS = PAGEDKV_POLY_PAIRS;
 constexpr int GROUP_BYTES = STEP * 128;  // one 64-dim column group of a 64-token K or V tile
 // D = head_dim (64, 128, 256); NT = row tiles per CTA (two tiles = two softmax warpgroups
 // taking turns on the tensor pipe and sharing the K/V rings).
@@ -1055,7 +1060,7 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
             (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
         // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
         // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
-        const double step_us = D == 256 ? 1.10 : D == 64 ? (nt == 1 ? 0.66 : 0.88) : (nt == 1 ? 0.80 : 0.86);
+        const double step_us = D == 256 ? 1.10 : D == 64 ? (nt == 1 ? 0.66 : 0.88) : (nt == 1 ? 0.65 : 0.84);
         const double unit_us = 8.0;
         auto consider = [&](int64_t T) {
             T = std::min(std::max<int64_t>(T, 1), steps_bound);
