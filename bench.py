@@ -195,7 +195,10 @@ def config_of(spec, world: int = 1, parallelism: str = ""):
 # dram__bytes_read.sum + dram__bytes_write.sum of one pa_decode_kernel launch, from the ncu
 # captures summarised under profiles/, keyed by (workload, H, Hkv, D, partition size the plan
 # chose).  Any other shape or partition size has no capture: null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    ("cfg3_fullpool_mixed_gqa", 32, 8, 128, 512): 1596370816,
+    ("cfg2_llama2_7b_mha", 32, 32, 128, 512): 1098308224,
+}
 
 
 def ncu_traffic(spec, partition_tokens: int):
