@@ -39,6 +39,7 @@ struct PlanParams {
     int batch;
     int max_blocks;
     int Hkv;
+    int H;              // query heads (rows per item that a split sequence sends to the combine)
     int forced_p;       // 0 = automatic
     int no_direct;      // 1 = every sequence goes through the combine kernel
     int64_t item_cap;   // records the workspace can hold
@@ -61,7 +62,9 @@ __device__ __forceinline__ int clamp_len(int L, int max_tok, bool& bad) {
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanParams p) {
-    __shared__ long long red[5][32];
+    // per warp: items for each candidate size, items of the forced size, then for each candidate
+    // the items of sequences that are split (their rows go through the combine) and the tokens
+    __shared__ long long red[10][32];
     __shared__ int s_P, s_bad;
     __shared__ int hist[MAX_PART / BS + 1], start[MAX_PART / BS + 1], cursor[MAX_PART / BS + 1];
     __shared__ int scan_warp[32];
@@ -77,16 +80,21 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     pdl_wait();               // the workspace may still be in use by the previous call
 
     // ---- pass 1: item counts for each candidate partition size ------------------------
-    long long cnt[5] = {0, 0, 0, 0, 0};
+    long long cnt[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     bool bad = false;
     for (int b = tid; b < p.batch; b += PLAN_THREADS) {
         const int L = clamp_len(p.seq_lens[b], max_tok, bad);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) cnt[c] += (L + cand[c] - 1) / cand[c];
+        for (int c = 0; c < 4; ++c) {
+            const int np = (L + cand[c] - 1) / cand[c];
+            cnt[c] += np;
+            if (np > 1) cnt[5 + c] += np;
+        }
         if (p.forced_p > 0) cnt[4] += (L + p.forced_p - 1) / p.forced_p;
+        cnt[9] += L;
     }
 #pragma unroll
-    for (int c = 0; c < 5; ++c) {
+    for (int c = 0; c < 10; ++c) {
         long long v = cnt[c];
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         if (lane == 0) red[c][warp] = v;
@@ -98,9 +106,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     if (warp == 0) {
         // lane w holds warp w's counts; one shuffle tree per candidate, every lane ends with
         // the totals
-        long long tot[5];
+        long long tot[10];
 #pragma unroll
-        for (int c = 0; c < 5; ++c) {
+        for (int c = 0; c < 10; ++c) {
             long long v = red[c][lane];
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
             tot[c] = v;
@@ -109,13 +117,22 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
         if (p.forced_p > 0) {
             P = tot[4] <= p.item_cap ? p.forced_p : 0;
         } else {
-            // walk from the largest partition down: stop as soon as every warp gets several
-            // units; never take a size whose items do not fit the workspace
-            const long long want = 4LL * p.total_warps;
+            // The size that minimises an estimate of the step, in KV tokens streamed by one
+            // warp: its share of all tokens (or one whole unit, when there are fewer units than
+            // warps), half a unit for the uneven end of the dynamic hand-out, and the combine --
+            // a partial row is about as many bytes as one token of one KV head, written and read
+            // back, at a quarter of the streaming efficiency.  Measured: workload 2 (64 sequences
+            // of at most 2048 tokens) is 3 % faster at 256 than at 512, workloads 3 and 5 (long
+            // sequences, many partials) 1.5 and 4 % slower.  Never a size whose items do not fit
+            // the workspace.
+            const float W = (float)p.total_warps;
+            const float share = (float)tot[9] * p.Hkv / W;
+            float best = 3.4e38f;
             for (int c = 3; c >= 0; --c) {
                 if (tot[c] > p.item_cap) break;
-                P = cand[c];
-                if (tot[c] * p.Hkv >= want) break;
+                const float Pc = (float)cand[c];
+                const float t = fmaxf(share, Pc) + 0.5f * Pc + 8.f * (float)tot[5 + c] * p.H / W;
+                if (t < best) best = t, P = cand[c];
             }
         }
         if (lane == 0) {
@@ -1070,6 +1087,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
         pp.batch = batch;
         pp.max_blocks = max_blocks_per_seq;
         pp.Hkv = shape->num_kv_heads;
+        pp.H = H;
         pp.forced_p = partition_tokens;
         pp.no_direct = part != nullptr;
         pp.item_cap = w.item_cap;
