@@ -197,7 +197,7 @@ def config_of(spec, world: int = 1, parallelism: str = ""):
 # chose).  Any other shape or partition size has no capture: null.
 NCU_TRAFFIC = {
     ("cfg3_fullpool_mixed_gqa", 32, 8, 128, 512): 1596370816,
-    ("cfg2_llama2_7b_mha", 32, 32, 128, 512): 1098308224,
+    ("cfg2_llama2_7b_mha", 32, 32, 128, 256): 1100236416,
 }
 
 
