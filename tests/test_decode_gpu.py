@@ -53,6 +53,19 @@ def test_head_layouts(H, Hkv, D):
         assert (out[6] == 0).all()
 
 
+def test_more_sequences_than_the_plan_kernel_has_threads():
+    # 2300 sequences: the plan walks them in three rounds of its 1024 threads, and only the
+    # first round's sequences have their lengths in the plan's shared memory; long sequences
+    # sit in every round so that split and unsplit rows come from both paths
+    rng = np.random.default_rng(5)
+    lens = rng.integers(0, 60, size=2300)
+    lens[[3, 1023, 1024, 1500, 2299]] = [700, 1300, 900, 2048, 513]
+    spec = wl.make_spec("t", seq_lens=lens, num_q_heads=4, num_kv_heads=2, head_dim=64,
+                        occupancy=0.95, seed=23)
+    for P in (0, 128):
+        run_and_check(spec, partition_tokens=P, what=f"2300 sequences P{P}")
+
+
 def test_many_short_and_ragged_sequences_span_all_warps():
     rng = np.random.default_rng(1)
     lens = rng.integers(0, 200, size=700)
