@@ -242,6 +242,27 @@ def test_pa_decode_host_reads_large_tables_in_place():
     assert int(g.status.item()) == 0
 
 
+@pytest.mark.parametrize("D,pinned", [(128, False), (256, True), (64, True)])
+def test_pa_decode_host_copies_what_it_cannot_read_in_place(D, pinned):
+    # pageable host tensors go through the device staging buffer (q always does); pinned
+    # tables and outputs of other head dims take the same call
+    spec = wl.make_spec("t", seq_lens=[40, 700, 0, 1300, 17], num_q_heads=8, num_kv_heads=2,
+                        head_dim=D, occupancy=0.9, seed=31 + D)
+    q, k, v = small_inputs(spec)
+    g = GpuDecode(spec, q, k, v)
+    dev_out = g.run().cpu()
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    qh, th, lh = pin(g.q.cpu()), pin(g.tables.cpu()), pin(g.lens.cpu())
+    oh = pin(torch.zeros_like(g.q.cpu()))
+    shape = api.shape_of(g.k, spec.num_q_heads)
+    io = torch.empty(api.pa_host_io_bytes(shape, spec.batch, th.shape[1]), dtype=torch.uint8,
+                     device="cuda")
+    api.pa_decode_host(qh, g.k, g.v, th, lh, spec.scale, oh, io, g.ws, dev_status=g.status)
+    torch.cuda.synchronize()
+    assert torch.equal(oh.view(torch.int16), dev_out.view(torch.int16))
+    assert int(g.status.item()) == 0
+
+
 def test_a_wait_that_nobody_completes_times_out_and_reports_it():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
