@@ -193,17 +193,17 @@ def config_of(spec, world: int = 1, parallelism: str = ""):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pa_decode_kernel launch, from the ncu
-# captures summarised under profiles/, keyed by (workload, H, Hkv, D, partition size the plan
-# chose).  Any other shape or partition size has no capture: null.
+# captures summarised under profiles/, keyed by (workload, context tokens, H, Hkv, D, partition
+# size the plan chose).  Any other size, shape or partition size has no capture: null.
 NCU_TRAFFIC = {
-    ("cfg3_fullpool_mixed_gqa", 32, 8, 128, 512): 1596370816,
-    ("cfg2_llama2_7b_mha", 32, 32, 128, 256): 1100236416,
+    ("cfg3_fullpool_mixed_gqa", 383921, 32, 8, 128, 512): 1596370816,
+    ("cfg2_llama2_7b_mha", 66297, 32, 32, 128, 256): 1100236416,
 }
 
 
 def ncu_traffic(spec, partition_tokens: int):
-    return NCU_TRAFFIC.get((spec.name, spec.num_q_heads, spec.num_kv_heads, spec.head_dim,
-                            int(partition_tokens)))
+    return NCU_TRAFFIC.get((spec.name, spec.total_tokens, spec.num_q_heads, spec.num_kv_heads,
+                            spec.head_dim, int(partition_tokens)))
 
 
 class DecodeLeg:

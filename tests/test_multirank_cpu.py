@@ -57,3 +57,33 @@ def test_reference_arm_prints_only_on_rank_zero():
     line = json.loads(r0.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_both_arms_describe_the_workload_with_the_same_config_object():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_07878_b200 import workloads as wl
+
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "1",
+           "--steps", "1", "--warmup", "0"]
+    r = subprocess.run(cmd, env=dict(os.environ, CUDA_VISIBLE_DEVICES=""), capture_output=True,
+                       text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["config"] == bench.config_of(wl.config_spec(1), 1)   # what the GPU arm prints
+
+
+def test_ncu_traffic_is_reported_only_for_the_captured_shape_and_partition_size():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_07878_b200 import workloads as wl
+
+    spec = wl.config_spec(3)
+    assert bench.ncu_traffic(spec, 512) == 1596370816
+    assert bench.ncu_traffic(spec, 256) is None
+    assert bench.ncu_traffic(wl.config_spec(3, scale_down=8), 512) is None   # same name, smaller
+    other = wl.make_spec(spec.name, seq_lens=spec.seq_lens, num_q_heads=16, num_kv_heads=8,
+                         head_dim=256, num_blocks=spec.num_blocks, seed=1)
+    assert bench.ncu_traffic(other, 512) is None
+    s = bench.spread([3.0, 1.0, 2.0])
+    assert (s["median"], s["min"], s["max"], s["n"]) == (2.0, 1.0, 3.0, 3)
