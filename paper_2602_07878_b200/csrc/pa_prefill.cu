@@ -279,7 +279,7 @@ static int launch_prefill(const CUtensorMap& km, const CUtensorMap& vm, const Pr
 // tcgen05 version: a row tile = 128 query rows ((token, head) pairs of one KV-head group)
 // ======================================================================================
 // Warps 0 .. 4 NT - 1: softmax and epilogue, four per tile (thread i of a tile's warps owns
-// row i = TMEM lane i); then one TMA producer warp and one MMA warp.  Per 64-token KV step and
+// row i = TMEM lane i); then four TMA producer warps and one MMA warp.  Per 64-token KV step and
 // tile: S = Q K^T (M 128, N 64, K head_dim) into one of two TMEM score buffers, the softmax
 // warps turn S into bf16 weights P written back over the first 32 columns of that score
 // buffer (and rescale the TMEM accumulator O when a row maximum has grown by more than 2^8),
