@@ -562,12 +562,19 @@ def e2e_leg(torch, api, leg, steps, repeats, dist):
     leg.step()
     torch.cuda.synchronize()
     assert torch.equal(oh.view(torch.int16), leg.out.cpu().view(torch.int16))
-    # q and lengths are copied; table entries are fetched in place over the link, once per
-    # (work item, KV head); output rows are posted in place
+    # lengths are copied; the query rows of a KV head's group (at most 8 heads per group, head_dim
+    # 64 or 128; otherwise q is copied once) and the table entries are fetched in place over the
+    # link, once per (work item, KV head); output rows are posted in place
     used_entries = int(((spec.seq_lens.astype(np.int64) + spec.block_size - 1) // spec.block_size).sum())
     table_bytes = th.numel() * 4
-    h2d = qh.numel() * 2 + lh.numel() * 4 + (used_entries * 4 * spec.num_kv_heads
-                                             if table_bytes >= (256 << 10) else table_bytes)
+    group = spec.num_q_heads // spec.num_kv_heads
+    units = leg.plan_header()["work_items"] * spec.num_kv_heads
+    q_in_place = units * group * spec.head_dim * 2
+    kv_us = spec.kv_bytes() / 6.4e6
+    q_bytes = (q_in_place if group <= 8 and spec.head_dim <= 128 and q_in_place / 50e3 <= 0.65 * kv_us
+               else qh.numel() * 2)   # the library's own rule for reading q in place
+    h2d = q_bytes + lh.numel() * 4 + (used_entries * 4 * spec.num_kv_heads
+                                      if table_bytes >= (256 << 10) else table_bytes)
     return regions, h2d, oh.numel() * 2
 
 

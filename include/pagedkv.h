@@ -232,11 +232,12 @@ int pa_host_io_bytes(const pa_shape* shape, int32_t max_batch, int32_t max_block
                      size_t* bytes);
 
 /*
- * pa_decode for a caller whose per-step tensors live in pinned host memory.  q_host and
- * seq_lens_host are copied to `io_buf` (dev, >= pa_host_io_bytes).  block_tables_host (if
- * 256 KiB or larger) and out_host are used in place when they are pinned memory the GPU can address (the kernels
- * then fetch table entries ahead of use and post output rows over the host link while they
- * run); otherwise they go through `io_buf` as well.  Everything is enqueued on
+ * pa_decode for a caller whose per-step tensors live in pinned host memory.  seq_lens_host is
+ * copied to `io_buf` (dev, >= pa_host_io_bytes).  q_host (groups of at most 8 query heads per KV
+ * head, head_dim 64 or 128), block_tables_host (if 256 KiB or larger) and out_host are used in
+ * place when they are pinned memory the GPU can address (the kernels then fetch query rows and
+ * table entries ahead of use and post output rows over the host link while they run);
+ * otherwise they go through `io_buf` as well.  Everything is enqueued on
  * `cuda_stream`; the KV cache itself stays on the device.  out_host is valid once the stream
  * has reached the end of this call, and the three host inputs must stay unchanged until then.
  */

@@ -275,9 +275,17 @@ struct UnitRegs {
     bool direct, valid, bad;
     int id;                                  // this lane's block id (block index = lane)
     uint32_t qa[D / 16][HI ? 4 : 2];         // A fragments of Q for every k-step
+    // q in host memory: the group's rows as fetched, 16 bytes per lane and piece (piece
+    // i * 32 + lane of the 8 x D block), turned into fragments when the unit becomes current
+    uint4 qraw[D / 32];
 };
 
-template <int D, bool HI, int NW, int NSLOT>
+// QH: q lives in pinned host memory (pa_decode_host).  Four-byte fragment loads would cross the
+// host link as 16-byte reads; the warp instead fetches the rows of a unit's head group with
+// 16-byte loads per lane (512 contiguous bytes per instruction), one unit ahead like the block
+// ids, and sorts them into fragments through a small shared-memory buffer.  At most 8 heads per
+// group and head_dim 64 or 128.
+template <int D, bool HI, int NW, int NSLOT, bool QH = false>
 __global__ void __launch_bounds__(NW * 32, 1)
 pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
                  const __grid_constant__ CUtensorMap vmap, const DecodeParams p) {
@@ -301,6 +309,8 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
     // instead of in a second set of registers, and fetched when that unit becomes current.
     constexpr bool QSTASH = D == 256;
     const uint32_t stash = base + NW * NSLOT * SLOT + NW * NSLOT * 8 + warp * (KS * QW * 128) + lane * 4;
+    static_assert(!QH || (!HI && D <= 128), "host q: groups of at most 8 heads, head_dim 64 or 128");
+    const uint32_t qrows = base + NW * NSLOT * SLOT + NW * NSLOT * 8 + warp * (8 * D * 2);  // QH only
 
     if (lane == 0) {
 #pragma unroll
@@ -351,6 +361,15 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         if (valid && lane < u.nblk)
             u.id = __ldg(&p.block_tables[(size_t)u.b * p.max_blocks + u.tok0 / BS + lane]);
         const size_t row0 = valid ? (size_t)u.b * p.q_stride + (size_t)kvh * G * D : 0;
+        if constexpr (QH) {
+            const uint4* q128 = reinterpret_cast<const uint4*>(p.q + row0);
+#pragma unroll
+            for (int i = 0; i < D / 32; ++i) {
+                const int piece = i * 32 + lane;           // 16-byte pieces of the 8 x D block
+                u.qraw[i] = valid && piece / (D / 8) < G ? __ldg(&q128[piece])
+                                                          : make_uint4(0u, 0u, 0u, 0u);
+            }
+        } else {
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
             // a0: (row g, k 2t..), a2: (row g, k 8+2t..); a1/a3 the same for row g+8
@@ -369,6 +388,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
                 else u.qa[ks][i] = w[i];
             }
         }
+        }
     };
     auto unpark = [&](Unit& u) {  // the parked fragments of the unit that has become current
 #pragma unroll
@@ -376,6 +396,22 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
 #pragma unroll
             for (int i = 0; i < QW; ++i)
                 asm volatile("ld.shared.b32 %0, [%1];" : "=r"(u.qa[ks][i]) : "r"(stash + (ks * QW + i) * 128));
+    };
+
+    auto unpark_host = [&](Unit& u) {  // QH: the rows fetched for this unit -> A fragments
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(qrows + (i * 32 + lane) * 16),
+                         "r"(u.qraw[i].x), "r"(u.qraw[i].y), "r"(u.qraw[i].z), "r"(u.qraw[i].w)
+                         : "memory");
+        __syncwarp();
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            const uint32_t a = qrows + (g * D + ks * 16 + 2 * t) * 2;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(u.qa[ks][0]) : "r"(a));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(u.qa[ks][QW - 1]) : "r"(a + 16));
+        }
+        __syncwarp();
     };
 
     Unit U0, U1;
@@ -392,6 +428,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         load_record(gw + 2 * total_warps, recB, kvhB, validB);
         if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
         build(r0, k0, v0, U0, false);
+        if (QH) unpark_host(U0);
         build(r1, k1, v1, U1, true);
     }
 
@@ -490,6 +527,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             // advance the fetch pipeline
             U0 = U1;
             if (QSTASH) unpark(U0);
+            if (QH) unpark_host(U0);
             build(recB, kvhB, validB, U1, true);
             const int w = __shfl_sync(0xffffffffu, wraw, 0);
             load_record(w, recB, kvhB, validB);
@@ -729,12 +767,13 @@ struct Variant {
     int nw, nslot;
 };
 
-template <int D, bool HI, int NW, int NSLOT>
+template <int D, bool HI, int NW, int NSLOT, bool QH = false>
 static int launch_decode(const CUtensorMap& km, const CUtensorMap& vm, const DecodeParams& dp,
                          const DeviceInfo& dev, int* grid_out, bool launch, cudaStream_t st) {
-    auto kern = pa_decode_kernel<D, HI, NW, NSLOT>;
-    // at head_dim 256 the Q fragments of the unit after the current one wait in shared memory
-    const int stash = D == 256 ? NW * (D / 16) * (HI ? 4 : 2) * 32 * 4 : 0;
+    auto kern = pa_decode_kernel<D, HI, NW, NSLOT, QH>;
+    // at head_dim 256 the Q fragments of the unit after the current one wait in shared memory;
+    // with q in host memory a warp sorts the fetched rows of a head group through 8 x D bf16
+    const int stash = D == 256 ? NW * (D / 16) * (HI ? 4 : 2) * 32 * 4 : QH ? NW * 8 * D * 2 : 0;
     const int smem = NW * NSLOT * (2 * BS * D * 2) + NW * NSLOT * 8 + stash + 1024;
     if (smem > dev.smem_optin) return PA_ERR_SHAPE;
     static int configured_dev = -1, ctas_per_sm = 0;
@@ -762,7 +801,11 @@ static int launch_decode(const CUtensorMap& km, const CUtensorMap& vm, const Dec
 template <int D, bool HI>
 static int dispatch_variant(Variant v, const CUtensorMap& km, const CUtensorMap& vm,
                             const DecodeParams& dp, const DeviceInfo& dev, int* warps, bool launch,
-                            cudaStream_t st) {
+                            cudaStream_t st, bool q_on_host) {
+    if constexpr (!HI && D <= 128) {
+        if (q_on_host)
+            return launch_decode<D, HI, 8, D == 64 ? 6 : 3, true>(km, vm, dp, dev, warps, launch, st);
+    }
     if constexpr (D == 256) {
         // a slot is 16 KiB: four warps with three slots each fill the shared memory
         return launch_decode<D, HI, 4, 3>(km, vm, dp, dev, warps, launch, st);
@@ -790,19 +833,25 @@ static Variant chosen_variant() {
     return v;
 }
 
+// q in host memory is read in place for groups of at most 8 heads at head_dim 64 or 128
+static bool host_q_supported(const pa_shape* s) {
+    return s->num_q_heads / s->num_kv_heads <= 8 && s->head_dim <= 128;
+}
+
 static int dispatch_decode(const pa_shape* s, const CUtensorMap& km, const CUtensorMap& vm,
                            const DecodeParams& dp, const DeviceInfo& dev, int* warps, bool launch,
-                           cudaStream_t st) {
+                           cudaStream_t st, bool q_on_host = false) {
     const bool hi = s->num_q_heads / s->num_kv_heads > 8;
     const Variant v = chosen_variant();
+    const bool qh = q_on_host && host_q_supported(s);
     if (s->head_dim == 256)
-        return hi ? dispatch_variant<256, true>(v, km, vm, dp, dev, warps, launch, st)
-                  : dispatch_variant<256, false>(v, km, vm, dp, dev, warps, launch, st);
+        return hi ? dispatch_variant<256, true>(v, km, vm, dp, dev, warps, launch, st, qh)
+                  : dispatch_variant<256, false>(v, km, vm, dp, dev, warps, launch, st, qh);
     if (s->head_dim == 128)
-        return hi ? dispatch_variant<128, true>(v, km, vm, dp, dev, warps, launch, st)
-                  : dispatch_variant<128, false>(v, km, vm, dp, dev, warps, launch, st);
-    return hi ? dispatch_variant<64, true>(v, km, vm, dp, dev, warps, launch, st)
-              : dispatch_variant<64, false>(v, km, vm, dp, dev, warps, launch, st);
+        return hi ? dispatch_variant<128, true>(v, km, vm, dp, dev, warps, launch, st, qh)
+                  : dispatch_variant<128, false>(v, km, vm, dp, dev, warps, launch, st, qh);
+    return hi ? dispatch_variant<64, true>(v, km, vm, dp, dev, warps, launch, st, qh)
+              : dispatch_variant<64, false>(v, km, vm, dp, dev, warps, launch, st, qh);
 }
 
 // ---- optional per-kernel timing (CUDA events recorded around each of the three launches) ----
@@ -1014,7 +1063,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
                        float scale, void* out, float* part, void* workspace,
                        size_t workspace_bytes, int32_t partition_tokens, int32_t flags,
                        int32_t* dev_status, void* cuda_stream, int64_t q_stride = 0,
-                       int64_t out_stride = 0) {
+                       int64_t out_stride = 0, bool q_on_host = false) {
     if (!shape) return PA_ERR_NULL;
     int rc = validate_shape(shape);
     if (rc) return rc;
@@ -1075,7 +1124,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     dp.out_stride = out_stride;
 
     int total_warps = 0;
-    rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, false, st);
+    rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, false, st, q_on_host);
     if (rc) return rc;
 
     ProfCall prof_ev;
@@ -1103,7 +1152,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     }
 
     if (prof) cudaEventRecord(prof_ev.ev[1], st);
-    rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, true, st);
+    rc = dispatch_decode(shape, km, vm, dp, dev, &total_warps, true, st, q_on_host);
     if (rc) return rc;
     if (prof) cudaEventRecord(prof_ev.ev[2], st);
 
@@ -1273,10 +1322,13 @@ extern "C" int pa_decode_host(const pa_shape* shape, const void* q_host, const v
     void* dtab = io + 2 * up(qbytes);
     void* dlen = io + 2 * up(qbytes) + up(tbytes);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    // Pinned memory the GPU can address is used in place: block-table entries are fetched two
-    // work units ahead of their use, and output rows are posted as they are produced, so both
-    // transfers overlap the kernels instead of preceding / following them.  q is re-read by
-    // every partition of a sequence and is copied once instead.
+    // Pinned memory the GPU can address is used in place: block-table entries and the query
+    // rows of a head group are fetched one to two work units ahead of their use (16 bytes per
+    // lane, so that they cross the link as whole 128-byte reads), and output rows are posted as
+    // they are produced: the transfers overlap the kernels instead of preceding / following
+    // them.  q is re-read by every (partition, KV head) unit, a few times its size over the
+    // link, which hides under the KV stream; groups of more than 8 heads and head_dim 256 copy
+    // it once instead.
     auto mapped = [](const void* host) -> void* {
         cudaPointerAttributes attr;
         if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
@@ -1289,8 +1341,33 @@ extern "C" int pa_decode_host(const pa_shape* shape, const void* q_host, const v
     void* tab_dev = tbytes >= (256u << 10) ? mapped(block_tables_host) : nullptr;
     void* out_dev = mapped(out_host);
     if (out_dev && (reinterpret_cast<uintptr_t>(out_dev) & 15)) out_dev = nullptr;
-    rc = check_cuda(cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, st));
-    if (rc) return rc;
+    void* q_dev = host_q_supported(shape) ? mapped(q_host) : nullptr;
+    if (q_dev && (reinterpret_cast<uintptr_t>(q_dev) & 15)) q_dev = nullptr;
+    if (q_dev) {
+        // Every (partition, KV head) unit fetches its group's rows: worth it only while those
+        // reads, at about 50 GB/s, fit well inside the time the KV stream takes at about
+        // 6.4 TB/s; a batch of long sequences with many query heads re-reads q tens of times
+        // and is better off with one copy.  The lengths are host data of this call.
+        const int64_t P = partition_tokens ? partition_tokens : MAX_PART;
+        const int64_t max_tok = (int64_t)max_blocks_per_seq * BS;
+        int64_t tokens = 0, items = 0;
+        for (int32_t b = 0; b < batch; ++b) {
+            const int64_t L = seq_lens_host[b];
+            if (L <= 0 || L > max_tok) continue;
+            tokens += L;
+            items += (L + P - 1) / P;
+        }
+        const int G = shape->num_q_heads / shape->num_kv_heads;
+        const double q_us = (double)items * shape->num_kv_heads * G * shape->head_dim * 2 / 50e3;
+        const double kv_us = (double)tokens * 2 * shape->num_kv_heads * shape->head_dim * 2 / 6.4e6;
+        if (q_us > 0.65 * kv_us) q_dev = nullptr;
+    }
+    const bool q_in_place = q_dev != nullptr;
+    if (!q_in_place) {
+        rc = check_cuda(cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, st));
+        if (rc) return rc;
+        q_dev = dq;
+    }
     if (!tab_dev) {
         rc = check_cuda(
             cudaMemcpyAsync(dtab, block_tables_host, tbytes, cudaMemcpyHostToDevice, st));
@@ -1300,10 +1377,10 @@ extern "C" int pa_decode_host(const pa_shape* shape, const void* q_host, const v
     rc = check_cuda(
         cudaMemcpyAsync(dlen, seq_lens_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st));
     if (rc) return rc;
-    rc = pa_decode(shape, dq, k_cache, v_cache, static_cast<const int32_t*>(tab_dev),
-                   max_blocks_per_seq, static_cast<const int32_t*>(dlen), batch, scale,
-                   out_dev ? out_dev : dout, workspace, workspace_bytes, partition_tokens, 0,
-                   dev_status, cuda_stream);
+    rc = decode_impl(shape, q_dev, k_cache, v_cache, static_cast<const int32_t*>(tab_dev),
+                     max_blocks_per_seq, static_cast<const int32_t*>(dlen), batch, scale,
+                     out_dev ? out_dev : dout, nullptr, workspace, workspace_bytes,
+                     partition_tokens, 0, dev_status, cuda_stream, 0, 0, q_in_place);
     if (rc || out_dev) return rc;
     return check_cuda(cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, st));
 }
