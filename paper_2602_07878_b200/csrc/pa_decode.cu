@@ -491,7 +491,31 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             const float l0 = A.l0, l1 = A.l1, m0 = A.m0, m1 = A.m1;
             auto& o = A.o;
             const int h0 = U0.kvh * G + g;
-            if (U0.direct) {
+            if (QH && U0.direct) {
+                // host-resident tensors: the rows go out as whole 16-byte pieces per lane (512
+                // contiguous bytes per instruction) instead of 4-byte fragments
+                const float i0 = U0.bad ? 0.f : 1.f / l0;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(qrows + (g * D + nt * 8 + 2 * t) * 2),
+                                 "r"(U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0))
+                                 : "memory");
+                __syncwarp();
+                uint4* orow = reinterpret_cast<uint4*>(p.out + (size_t)U0.b * p.out_stride +
+                                                       (size_t)U0.kvh * G * D);
+#pragma unroll
+                for (int i = 0; i < D / 32; ++i) {
+                    const int piece = i * 32 + lane;
+                    if (piece / (D / 8) < G) {
+                        uint4 w;
+                        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                                     : "r"(qrows + piece * 16));
+                        orow[piece] = w;
+                    }
+                }
+                __syncwarp();
+            } else if (U0.direct) {
                 const float i0 = U0.bad ? 0.f : 1.f / l0, i1 = U0.bad ? 0.f : 1.f / l1;
                 if (g < G) {
                     uint32_t* dst = reinterpret_cast<uint32_t*>(
