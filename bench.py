@@ -725,19 +725,32 @@ def run_ours(args):
                                                 args.recompute_chunk, args.recompute_split,
                                                 shape=rshape, cpu=not args.no_cpu,
                                                 clock_ms=args.recompute_clock_ms)
+        def resources(fn):
+            """A leg that cannot get its memory (device pool, gigabytes of pinned host memory)
+            is reported as skipped; a library error or a failed check still ends the run."""
+            try:
+                return fn()
+            except api.PagedKVError:
+                raise
+            except RuntimeError as exc:   # torch: out of device memory, pinning failed
+                torch.cuda.empty_cache()
+                return {"skipped": f"{type(exc).__name__}: {str(exc)[:160]}"}
+
         if not args.no_swap:
-            line["swap"] = bench_swap(args, torch, api, wl, leg.step, leg.step_bytes)
+            line["swap"] = resources(lambda: bench_swap(args, torch, api, wl, leg.step, leg.step_bytes))
         if not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(args, spec, leg.q, leg.k, leg.v)
         if not args.no_workloads:
-            line["workloads"] = workloads_object(torch, api, wl, args, args.workload)
+            line["workloads"] = resources(lambda: workloads_object(torch, api, wl, args, args.workload))
             # workload 4 at full size needs 126 GB of pool and 8 GiB of pinned host memory:
             # release everything else first, then run it if the device has the room
             del leg
             torch.cuda.empty_cache()
             free, _ = torch.cuda.mem_get_info()
-            if free >= 150 * (1 << 30):
-                line["workloads"]["cfg4_swap_churn"] = churn_leg(args, torch, api, wl)
+            if "skipped" in line["workloads"]:
+                pass
+            elif free >= 150 * (1 << 30):
+                line["workloads"]["cfg4_swap_churn"] = resources(lambda: churn_leg(args, torch, api, wl))
             else:
                 line["workloads"]["cfg4_swap_churn"] = {
                     "skipped": f"{free / 2**30:.0f} GiB free on the device, 150 GiB wanted "
