@@ -81,6 +81,31 @@ def test_full_size_decode_sampled_against_oracle(index, n_long, n_other):
     assert_parity(torch_to_f64(out[seqs]), ref, spec.name)
 
 
+@pytest.mark.parametrize("index", [2, 3, 5])
+def test_full_size_host_call_gives_the_device_call_bits(index):
+    # pa_decode_host at the bench's sizes: workloads 2 and 3 read q in place from pinned host
+    # memory (the host-memory instantiation of the attention kernel), workload 5 copies it
+    spec = wl.config_spec(index)
+    k, v = wl.pools_torch(spec, "cuda")
+    q, out, hdr = decode_full(spec, k, v)
+    tables = torch.from_numpy(spec.block_tables).pin_memory()
+    lens = torch.from_numpy(spec.seq_lens).pin_memory()
+    qh = q.cpu().pin_memory()
+    oh = torch.zeros_like(qh).pin_memory()
+    shape = api.shape_of(k, spec.num_q_heads)
+    io = torch.empty(api.pa_host_io_bytes(shape, spec.batch, tables.shape[1]), dtype=torch.uint8,
+                     device="cuda")
+    ws = torch.empty(api.pa_workspace_bytes(shape, spec.batch, spec.total_tokens + 16 * spec.batch),
+                     dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(2):
+        oh.zero_()
+        api.pa_decode_host(qh, k, v, tables, lens, spec.scale, oh, io, ws, dev_status=status)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+    assert int(status.item()) == 0
+
+
 def test_full_size_swap_churn_and_decode():
     """Workload 4 at full size: 32-layer pool of 60000 blocks at 98 % occupancy; evict 64K
     tokens' worth of whole sequences, restore them into other blocks, decode one layer."""
