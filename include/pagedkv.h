@@ -355,8 +355,13 @@ int kv_block_bytes(const kv_pool_desc* pool, const pa_shape* shape, size_t* byte
  *   pinned_host_buf  pinned host memory, 16-byte aligned, >= n * kv_block_bytes
  *   staging          dev scratch or NULL.  With a staging buffer (any size >= one block
  *                    image, 256-byte aligned) blocks are gathered into it by a kernel and
- *                    moved by the copy engine in pieces of staging_bytes; with NULL the
- *                    gather kernel stores straight into the pinned buffer.
+ *                    moved by the copy engine; with NULL the gather kernel stores straight
+ *                    into the pinned buffer.  A swap larger than the staging buffer is moved
+ *                    in pieces that alternate between the buffer's two halves (each at least
+ *                    one block image), the copy of one piece running beside the gather of
+ *                    the next: for the length of such a call the library creates a side
+ *                    stream and four events, tied to `cuda_stream` by event waits and
+ *                    destroyed before the call returns.
  * The image is complete when `cuda_stream` reaches the end of the call.
  */
 int kv_swap_out(const kv_pool_desc* pool, const pa_shape* shape, const void* k_pool,

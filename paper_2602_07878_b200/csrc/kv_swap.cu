@@ -120,14 +120,77 @@ static int swap_common(const SwapCall& c, bool out) {
     p.log2_d = s.head_dim == 256 ? 8 : s.head_dim == 128 ? 7 : 6;
     p.vec_per_chunk = (int)(chunk_bytes / 16);
 
-    for (int32_t done = 0; done < c.n; done += per_launch) {
+    // Staged swaps of more than one piece alternate between the two halves of the staging
+    // buffer: the copy engine moves one half over the link (on a side stream that lives for
+    // this call only) while the kernel gathers into, or scatters from, the other.  Events tie
+    // the two streams together, and everything joins the caller's stream before the call
+    // returns, so the caller sees ordinary stream order.
+    const bool two_halves = c.staging && c.n > per_launch && c.staging_bytes / 2 >= block_bytes;
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_kernel[2] = {nullptr, nullptr}, ev_copy[2] = {nullptr, nullptr};
+    auto cleanup = [&]() {
+        for (int h = 0; h < 2; ++h) {
+            if (ev_kernel[h]) cudaEventDestroy(ev_kernel[h]);
+            if (ev_copy[h]) cudaEventDestroy(ev_copy[h]);
+        }
+        if (side) cudaStreamDestroy(side);  // work already queued on it still completes
+    };
+    size_t half_bytes = 0;
+    if (two_halves) {
+        half_bytes = (c.staging_bytes / 2) & ~(size_t)255;
+        per_launch = (int)std::min<size_t>(SWAP_IDS, half_bytes / block_bytes);
+        rc = check_cuda(cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking));
+        for (int h = 0; h < 2 && !rc; ++h) {
+            rc = check_cuda(cudaEventCreateWithFlags(&ev_kernel[h], cudaEventDisableTiming));
+            if (!rc) rc = check_cuda(cudaEventCreateWithFlags(&ev_copy[h], cudaEventDisableTiming));
+        }
+        if (rc) {
+            cleanup();
+            return rc;
+        }
+    }
+
+    int piece = 0;
+    for (int32_t done = 0; done < c.n; done += per_launch, ++piece) {
         const int m = std::min<int32_t>(per_launch, c.n - done);
         SwapIds ids;
         for (int i = 0; i < m; ++i) ids.v[i] = c.ids[done + i];
         const size_t bytes = block_bytes * (size_t)m;
         uint8_t* host_piece = c.host + block_bytes * (size_t)done;
         const unsigned grid = (unsigned)m * p.layers * 2;
-        if (c.staging) {
+        if (two_halves) {
+            const int h = piece & 1;
+            uint8_t* half = c.staging + (size_t)h * half_bytes;
+            p.image = half;
+            if (out) {
+                // the half is free once the copy that emptied it two pieces ago has finished
+                if (piece >= 2) rc = check_cuda(cudaStreamWaitEvent(c.st, ev_copy[h], 0));
+                if (rc) break;
+                kv_swap_kernel<true><<<grid, SWAP_THREADS, 0, c.st>>>(p, ids);
+                count_launch();
+                rc = check_cuda(cudaGetLastError());
+                if (!rc) rc = check_cuda(cudaEventRecord(ev_kernel[h], c.st));
+                if (!rc) rc = check_cuda(cudaStreamWaitEvent(side, ev_kernel[h], 0));
+                if (!rc) rc = check_cuda(cudaMemcpyAsync(host_piece, half, bytes, cudaMemcpyDeviceToHost, side));
+                if (!rc) rc = check_cuda(cudaEventRecord(ev_copy[h], side));
+            } else {
+                // the first copies wait for whatever the caller's stream did before this call
+                // (the staging buffer may still be in use); later ones for the scatter kernel
+                // that read the half two pieces ago
+                if (piece < 2) {
+                    rc = check_cuda(cudaEventRecord(ev_kernel[h], c.st));
+                }
+                if (!rc) rc = check_cuda(cudaStreamWaitEvent(side, ev_kernel[h], 0));
+                if (!rc) rc = check_cuda(cudaMemcpyAsync(half, host_piece, bytes, cudaMemcpyHostToDevice, side));
+                if (!rc) rc = check_cuda(cudaEventRecord(ev_copy[h], side));
+                if (!rc) rc = check_cuda(cudaStreamWaitEvent(c.st, ev_copy[h], 0));
+                if (rc) break;
+                kv_swap_kernel<false><<<grid, SWAP_THREADS, 0, c.st>>>(p, ids);
+                count_launch();
+                rc = check_cuda(cudaGetLastError());
+                if (!rc) rc = check_cuda(cudaEventRecord(ev_kernel[h], c.st));
+            }
+        } else if (c.staging) {
             p.image = c.staging;
             if (out) {
                 kv_swap_kernel<true><<<grid, SWAP_THREADS, 0, c.st>>>(p, ids);
@@ -153,8 +216,19 @@ static int swap_common(const SwapCall& c, bool out) {
             count_launch();
             rc = check_cuda(cudaGetLastError());
         }
-        if (rc) return rc;
+        if (rc) break;
     }
+    if (two_halves) {
+        // the caller's stream continues only after the last copies of a swap-out have landed
+        // (for a swap-in its own scatter kernels already come after every copy)
+        if (out)
+            for (int h = 0; h < 2 && h < piece; ++h) {
+                const int rc2 = check_cuda(cudaStreamWaitEvent(c.st, ev_copy[h], 0));
+                if (!rc) rc = rc2;
+            }
+        cleanup();
+    }
+    if (rc) return rc;
     return PA_OK;
 }
 
