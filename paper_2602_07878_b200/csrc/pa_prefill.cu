@@ -1056,8 +1056,13 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
     for (int nt = 1; nt <= (D == 256 ? 1 : 2); ++nt) {  // head_dim 256: one tile fills the TMEM
         if (forced_tiles && nt != forced_tiles && D != 256) continue;
         const int64_t tpg = (int64_t)nt * tpt;
+        // row groups: exact for one sequence; for several, as if they shared the query tokens
+        // evenly (a batch of short chunks leaves the second tile of a two-tile CTA empty),
+        // never more than the bound the grid is sized with
+        const int64_t avg_q = (total_q + batch - 1) / batch;
         const int64_t groups =
-            (batch == 1 ? (total_q + tpg - 1) / tpg : total_q / tpg + batch) * Hkv;
+            (batch == 1 ? (total_q + tpg - 1) / tpg
+                        : std::min<int64_t>(total_q / tpg + batch, batch * ((avg_q + tpg - 1) / tpg))) * Hkv;
         // measured on 512-token chunks at 2K..32K context: microseconds per 64-token step of a
         // CTA, per unit (set-up, pipeline fill, epilogue), and per byte of partial records
         const double step_us = D == 256 ? 1.10 : D == 64 ? (nt == 1 ? 0.66 : 0.88) : (nt == 1 ? 0.65 : 0.84);
@@ -1082,11 +1087,14 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
             continue;
         }
         // even splits, and split lengths in between (a short last split fills SMs that a
-        // whole number of equal units would leave idle)
-        for (int64_t S = 1; S <= std::max<int64_t>(1, std::min<int64_t>(cap_fit, 64)); ++S)
-            consider((steps_bound + S - 1) / S);
-        if (cap_fit > 1)
+        // whole number of equal units would leave idle); a context too short to give every
+        // split its 8 steps is looked at once (small calls are bound by the host's issue rate)
+        const int64_t s_hi = std::min<int64_t>({cap_fit, 64, steps_bound / 8});
+        consider(steps_bound);
+        if (s_hi > 1) {
+            for (int64_t S = 2; S <= s_hi; ++S) consider((steps_bound + S - 1) / S);
             for (int64_t i = 1; i < 48; ++i) consider(steps_bound * i / 48);
+        }
     }
     return best;
 }

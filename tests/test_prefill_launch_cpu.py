@@ -77,3 +77,12 @@ def test_more_sms_never_means_fewer_units():
         units = -(-512 // (tiles * 32)) * 8 * splits
         assert units >= prev
         prev = units
+
+
+def test_a_batch_of_short_chunks_takes_one_tile_per_cta():
+    # 64 sequences of 8 query tokens each (32 / 8 heads: 32 tokens fill a 128-row tile): a
+    # second tile per CTA would stay empty, so one tile it is; four sequences of 128 tokens
+    # fill two tiles each
+    sh = shape(32, 8, 128)
+    assert api.pa_prefill_select_launch(sh, 64, 512, 32, ws(sh, 64, 512, 4))[0] == 1
+    assert api.pa_prefill_select_launch(sh, 4, 512, 256, ws(sh, 4, 512, 4))[0] == 2
