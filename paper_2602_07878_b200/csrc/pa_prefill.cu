@@ -878,6 +878,19 @@ __global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMerg
     pdl_wait();
     if (n_vis == 0) return;
     const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + (size_t)row * p.split_cap;
+    const float4* po = reinterpret_cast<const float4*>(p.part_o) + (size_t)row * p.split_cap * (D / 4);
+    // the usual case, two to four splits: every row of every split is requested before the
+    // first weight is known, so the (exponent, sum) pairs and the rows share one round trip
+    const bool few = n_vis <= 4;
+    float4 o[4][NV];
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c = lane + 32 * v;
+            o[s][v] = few && s < n_vis && c < D / 4 ? po[(size_t)s * (D / 4) + c]
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
     float M = -INFINITY;
     bool bad = false;
     for (int s = lane; s < n_vis; s += 32) {
@@ -887,11 +900,26 @@ __global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMerg
     }
     for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     bad = __any_sync(0xffffffffu, bad);
-    const float4* po = reinterpret_cast<const float4*>(p.part_o) + (size_t)row * p.split_cap * (D / 4);
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     float lsum = 0.f;
+    if (few) {
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            if (s >= n_vis) break;
+            const float2 v2 = ml[s];
+            const float w = v2.x == -INFINITY ? 0.f : ex2(v2.x - M);
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                acc[v].x = fmaf(w, o[s][v].x, acc[v].x);
+                acc[v].y = fmaf(w, o[s][v].y, acc[v].y);
+                acc[v].z = fmaf(w, o[s][v].z, acc[v].z);
+                acc[v].w = fmaf(w, o[s][v].w, acc[v].w);
+            }
+            lsum = fmaf(w, v2.y, lsum);
+        }
+    } else
 #pragma unroll 4
     for (int s = 0; s < n_vis; ++s) {
         const float2 v2 = ml[s];
