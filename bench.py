@@ -895,6 +895,24 @@ def bench_probes(torch, api, copy_peak, step_gbps, kernel_gbps, gib=2, reps=5):
             e1.synchronize()
             best = max(best, buf.numel() / e0.elapsed_time(e1) / 1e6)
         out[name] = best
+    # how fast 2 KB tiled TMA boxes (the K/V box of the attention kernels) can be issued and
+    # delivered out of L2: a 64 MiB buffer walked 32 times, 16 boxes per SM and ring slot,
+    # issued by 1, 2, 4 or 8 warps
+    small = buf[:64 << 20]
+    clock_hz = 1.965e9
+    rows = []
+    for warps, boxes in ((1, 16), (2, 8), (4, 4), (8, 2)):
+        api.pa_probe_tma_issue(small, warps, boxes, 2, status)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        n = api.pa_probe_tma_issue(small, warps, boxes, 32, status)
+        e1.record()
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        rows.append({"warps": warps, "boxes_per_instruction": boxes, "gbps": n * 2048 / ms / 1e6,
+                     "ns_per_box_per_sm": ms * 1e6 / (n / 148.0),
+                     "bytes_per_clock_per_sm_at_1965mhz": n * 2048 / 148.0 / (ms * 1e-3 * clock_hz)})
+    out["tma_issue_l2_resident"] = rows
     assert int(status.item()) == 0
     out["attention_kernel_frac_of_gather"] = kernel_gbps / out["read_gather_4k_gbps"]
     out["step_frac_of_gather"] = step_gbps / out["read_gather_4k_gbps"]

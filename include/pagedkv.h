@@ -403,6 +403,21 @@ int pa_probe_read(const void* dev_buf, size_t bytes, int32_t scattered, uint32_t
                   void* dev_sink, int32_t* dev_status, void* cuda_stream);
 
 /*
+ * Issue-rate probe for tiled TMA loads (no counterpart in the paper; a measurement aid behind
+ * the choice of four producer warps in the prefill kernel).  `dev_buf` (256-byte aligned, 64 KiB
+ * to 2 GiB, whole multiples of 32 KiB are used) is viewed as [blocks][8][16][128] bf16; on every
+ * SM `warps` warps (1..8) each keep six ring slots in flight and issue, per slot, `boxes` boxes
+ * of 2 KB (64 dims x 16 tokens: the K/V box of the attention kernels) from as many lanes of one
+ * instruction (`boxes` even, 2..16, warps * boxes <= 16), walking the buffer `reps` times.  With
+ * a buffer that fits L2 the elapsed time measures how fast boxes can be issued and delivered.
+ * *boxes_issued (host, may be NULL) receives the number of boxes the launch issues in total.
+ * dev_status gets PA_STATUS_TIMEOUT if a bounded wait gives up.
+ */
+int pa_probe_tma_issue(const void* dev_buf, size_t bytes, int32_t warps, int32_t boxes,
+                       int32_t reps, int64_t* boxes_issued, int32_t* dev_status,
+                       void* cuda_stream);
+
+/*
  * Self-test of the bounded waits (no counterpart in the paper).  Every wait inside the
  * kernels (on TMA data, on tensor-core completion, on another warp) gives up after a wall-
  * clock limit, reports PA_STATUS_TIMEOUT and lets the kernel return, so that a lost signal

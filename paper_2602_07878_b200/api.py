@@ -33,7 +33,7 @@ EXPORTS = ["pa_workspace_bytes", "pa_decode", "pa_decode_strided", "pa_host_io_b
            "pa_decode_static", "kv_append", "pa_partial_floats", "pa_decode_partial",
            "pa_merge_partials",
            "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_split",
-           "pa_prefill_split_workspace_bytes", "pa_prefill_last_launch", "pa_prefill_select_launch", "pa_selftest_wait_expiry", "pa_probe_read"]
+           "pa_prefill_split_workspace_bytes", "pa_prefill_last_launch", "pa_prefill_select_launch", "pa_selftest_wait_expiry", "pa_probe_read", "pa_probe_tma_issue"]
 
 
 class PaShape(ctypes.Structure):
@@ -103,6 +103,8 @@ def lib() -> ctypes.CDLL:
         L.pa_selftest_wait_expiry.restype = ctypes.c_int
         L.pa_probe_read.argtypes = [vp, sz, i32, ctypes.c_uint32, vp, vp, vp]
         L.pa_probe_read.restype = ctypes.c_int
+        L.pa_probe_tma_issue.argtypes = [vp, sz, i32, i32, i32, ctypes.POINTER(ctypes.c_int64), vp, vp]
+        L.pa_probe_tma_issue.restype = ctypes.c_int
         L.kv_append.argtypes = [pshape, vp, vp, vp, vp, vp, i32, vp, vp]
         L.kv_append.restype = ctypes.c_int
         L.pa_decode_strided.argtypes = [pshape, vp, ctypes.c_int64, vp, vp, vp, i32, vp, i32,
@@ -435,6 +437,15 @@ def pa_selftest_wait_expiry(limit_us: int, dev_status, stream=None):
     """Forward to pa_selftest_wait_expiry: a bounded wait that must run out and report it."""
     _check(lib().pa_selftest_wait_expiry(int(limit_us), _ptr(dev_status), _stream(stream)),
            "pa_selftest_wait_expiry")
+
+
+def pa_probe_tma_issue(buf, warps: int, boxes: int, reps: int, dev_status, stream=None) -> int:
+    """Forward to pa_probe_tma_issue; returns the number of 2 KB boxes the launch issues."""
+    n = ctypes.c_int64(0)
+    _check(lib().pa_probe_tma_issue(_ptr(buf), buf.numel() * buf.element_size(), warps, boxes, reps,
+                                    ctypes.byref(n), _ptr(dev_status), _stream(stream)),
+           "pa_probe_tma_issue")
+    return int(n.value)
 
 
 def pa_probe_read(buf, scattered: bool, dev_status, seed: int = 1, stream=None):

@@ -326,9 +326,10 @@ struct Cfg {
     static constexpr int TMEM_COLS = NT * TILE_COLS <= 256 ? 256 : 512;
     static_assert(NT * TILE_COLS <= 512, "tensor memory holds 512 columns");
     static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
-    // Four TMA producer warps, one per 16-token block of a step: a warp pays some 400 cycles
-    // per bulk-tensor instruction plus about 45 per lane that issues a box in it, so one warp
-    // issuing the 16 boxes (2 KB each) of a head_dim-128 step cannot keep up with the MMAs.
+    // Four TMA producer warps, one per 16-token block of a step: a single warp delivers a 2 KB
+    // box about every 85 cycles however many are in flight (pa_probe_tma_issue), so one warp
+    // issuing the 16 boxes of a head_dim-128 step cannot keep up with the MMAs; four warps
+    // with four boxes each take half the time.
     static constexpr int N_PRODUCERS = 4;
     static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + N_PRODUCERS,
                          THREADS = (4 * NT + N_PRODUCERS + 1) * 32;

@@ -118,3 +118,17 @@ def test_swap_argument_errors_return_before_any_launch(L):
     assert L.kv_swap_in(ctypes.byref(pool), ctypes.byref(s), A, A, A, 3 * bb.value, ids, 3,
                         None, 0, None) == api.ERR["BLOCK_ID"]
     assert L.pa_launch_count() == n0
+
+
+def test_tma_issue_probe_refuses_bad_shapes_before_any_launch():
+    import ctypes
+    L = api.lib()
+    n = ctypes.c_int64(0)
+    buf, st = ctypes.c_void_p(1 << 20), ctypes.c_void_p(256)      # never dereferenced on the host
+    call = lambda warps, boxes, reps=1, nbytes=1 << 20: L.pa_probe_tma_issue(
+        buf, nbytes, warps, boxes, reps, ctypes.byref(n), st, None)
+    assert call(0, 2) == api.ERR["ARG"] and call(9, 2) == api.ERR["ARG"]
+    assert call(1, 3) == api.ERR["ARG"] and call(1, 18) == api.ERR["ARG"]
+    assert call(8, 4) == api.ERR["ARG"]            # 32 boxes per slot round do not fit the rings
+    assert call(1, 2, 0) == api.ERR["ARG"] and call(1, 2, 1, 1 << 10) == api.ERR["ARG"]
+    assert L.pa_probe_tma_issue(None, 1 << 20, 1, 2, 1, None, st, None) == api.ERR["NULL"]

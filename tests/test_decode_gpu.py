@@ -287,3 +287,15 @@ def test_read_probes_run_and_report_no_timeout():
     api.pa_probe_read(buf[: 4096 * 3], True, status)      # fewer granules than warps
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and api.pa_launch_count() - n0 == 3
+
+
+@pytest.mark.parametrize("warps,boxes", [(1, 16), (4, 4), (8, 2), (2, 2)])
+def test_tma_issue_probe_runs_and_counts_its_boxes(warps, boxes):
+    buf = torch.zeros(8 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n = api.pa_probe_tma_issue(buf, warps, boxes, 3, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # every warp of every SM issues the same number of slots; the whole buffer is covered 3 times
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert n % (sms * warps * boxes) == 0 and n * 2048 >= 3 * buf.numel()
