@@ -72,7 +72,7 @@ typedef struct pa_shape {
     int32_t num_kv_heads; /* Hkv                                                           */
     int32_t head_dim;     /* D: 64, 128 or 256                                             */
     int32_t block_size;   /* tokens per block: 16                                          */
-    int32_t num_blocks;   /* physical pool size                                            */
+    int32_t num_blocks;   /* physical pool size, at least 1                                */
     int32_t dtype;        /* PA_BF16                                                       */
     int64_t stride_block;
     int64_t stride_head;

@@ -247,7 +247,7 @@ def _build_tables(seq_lens: np.ndarray, block_size: int, num_blocks: int,
 
 def _pool_for_occupancy(seq_lens, block_size, occupancy):
     nb = int(((seq_lens.astype(np.int64) + block_size - 1) // block_size).sum())
-    return int(math.ceil(nb / occupancy))
+    return max(1, int(math.ceil(nb / occupancy)))   # a pool has at least one block
 
 
 def make_spec(name: str, *, seq_lens, num_q_heads, num_kv_heads, head_dim, block_size=16,

@@ -299,3 +299,12 @@ def test_tma_issue_probe_runs_and_counts_its_boxes(warps, boxes):
     # every warp of every SM issues the same number of slots; the whole buffer is covered 3 times
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     assert n % (sms * warps * boxes) == 0 and n * 2048 >= 3 * buf.numel()
+
+
+def test_a_batch_of_empty_sequences_gives_zero_rows():
+    # nothing allocated at all: the pool still has a block, every output row is zeros
+    spec = wl.make_spec("t", seq_lens=[0, 0, 0], num_q_heads=8, num_kv_heads=8, head_dim=64,
+                        occupancy=1.0, seed=3)
+    assert spec.num_blocks == 1
+    _, g, out, ref = run_and_check(spec)
+    assert (out == 0).all() and int(g.status.item()) == 0
