@@ -6,7 +6,10 @@
 
 namespace pk {
 
-template <int D, bool HI>
+// SPLITW: each softmax weight goes to the MMA as two bf16 numbers, its rounded value and the
+// rounded remainder, so the weights carry about 16 significant bits and the result differs
+// from the exact weighted mean by the output's own rounding only.  It doubles the P V MMAs.
+template <int D, bool HI, bool SPLITW = false>
 struct AttnFrag {
     static constexpr int KS = D / 16;      // k-steps of Q K^T
     static constexpr int NT = D / 8;       // n-tiles of O
@@ -84,11 +87,20 @@ struct AttnFrag {
         const float mu0 = mn0 == -INFINITY ? 0.f : mn0;
         const float corr0 = ex2(m0 - mu0);
         m0 = mn0;
-        const uint32_t pa0 = pack_bf16x2(ex2(s0[0] - mu0), ex2(s0[1] - mu0));
-        const uint32_t pa2 = pack_bf16x2(ex2(s1[0] - mu0), ex2(s1[1] - mu0));
-        // the row sum uses the rounded weights, the same ones the MMA multiplies by
-        l0 = l0 * corr0 + ((bf16lo_to_f32(pa0) + bf16hi_to_f32(pa0)) +
-                           (bf16lo_to_f32(pa2) + bf16hi_to_f32(pa2)));
+        const float e00 = ex2(s0[0] - mu0), e01 = ex2(s0[1] - mu0);
+        const float e10 = ex2(s1[0] - mu0), e11 = ex2(s1[1] - mu0);
+        const uint32_t pa0 = pack_bf16x2(e00, e01);
+        const uint32_t pa2 = pack_bf16x2(e10, e11);
+        uint32_t pb0 = 0u, pb1 = 0u, pb2 = 0u, pb3 = 0u;
+        if (SPLITW) {
+            pb0 = pack_bf16x2(e00 - bf16lo_to_f32(pa0), e01 - bf16hi_to_f32(pa0));
+            pb2 = pack_bf16x2(e10 - bf16lo_to_f32(pa2), e11 - bf16hi_to_f32(pa2));
+            l0 = l0 * corr0 + ((e00 + e01) + (e10 + e11));
+        } else {
+            // the row sum uses the rounded weights, the same ones the MMA multiplies by
+            l0 = l0 * corr0 + ((bf16lo_to_f32(pa0) + bf16hi_to_f32(pa0)) +
+                               (bf16lo_to_f32(pa2) + bf16hi_to_f32(pa2)));
+        }
         uint32_t pa1 = 0u, pa3 = 0u;
         float corr1 = 1.f;
         if (HI) {
@@ -103,10 +115,18 @@ struct AttnFrag {
             const float mu1 = mn1 == -INFINITY ? 0.f : mn1;
             corr1 = ex2(m1 - mu1);
             m1 = mn1;
-            pa1 = pack_bf16x2(ex2(s0[2] - mu1), ex2(s0[3] - mu1));
-            pa3 = pack_bf16x2(ex2(s1[2] - mu1), ex2(s1[3] - mu1));
-            l1 = l1 * corr1 + ((bf16lo_to_f32(pa1) + bf16hi_to_f32(pa1)) +
-                               (bf16lo_to_f32(pa3) + bf16hi_to_f32(pa3)));
+            const float f00 = ex2(s0[2] - mu1), f01 = ex2(s0[3] - mu1);
+            const float f10 = ex2(s1[2] - mu1), f11 = ex2(s1[3] - mu1);
+            pa1 = pack_bf16x2(f00, f01);
+            pa3 = pack_bf16x2(f10, f11);
+            if (SPLITW) {
+                pb1 = pack_bf16x2(f00 - bf16lo_to_f32(pa1), f01 - bf16hi_to_f32(pa1));
+                pb3 = pack_bf16x2(f10 - bf16lo_to_f32(pa3), f11 - bf16hi_to_f32(pa3));
+                l1 = l1 * corr1 + ((f00 + f01) + (f10 + f11));
+            } else {
+                l1 = l1 * corr1 + ((bf16lo_to_f32(pa1) + bf16hi_to_f32(pa1)) +
+                                   (bf16lo_to_f32(pa3) + bf16hi_to_f32(pa3)));
+            }
         }
         // rescale only when some row's maximum moved (warp-uniform branch)
         if (__any_sync(0xffffffffu, corr0 != 1.f || corr1 != 1.f)) {
@@ -130,6 +150,10 @@ struct AttnFrag {
                               v3);
             mma_bf16_16816(o[2 * jj], pa0, pa1, pa2, pa3, v0, v1);
             mma_bf16_16816(o[2 * jj + 1], pa0, pa1, pa2, pa3, v2, v3);
+            if (SPLITW) {
+                mma_bf16_16816(o[2 * jj], pb0, pb1, pb2, pb3, v0, v1);
+                mma_bf16_16816(o[2 * jj + 1], pb0, pb1, pb2, pb3, v2, v3);
+            }
         }
     }
 

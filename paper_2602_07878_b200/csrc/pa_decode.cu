@@ -432,7 +432,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         build(r1, k1, v1, U1, true);
     }
 
-    AttnFrag<D, HI> A;
+    AttnFrag<D, HI, true> A;
     A.init_lane(lane);
     A.reset();
 

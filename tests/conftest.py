@@ -38,7 +38,10 @@ def pytest_terminal_summary(terminalreporter, exitstatus, config):
     terminalreporter.write_line(
         f"parity tally: {t['calls']} comparisons with the oracle, {t['elements']} elements "
         f"({t['amended_elements']} of them prefill outputs under the amended bound); "
-        f"{t['over_abs_tol']} elements above 1e-2"
+        f"decode: {t['decode_over_abs_tol']} of {t['decode_elements']} elements above 1e-2"
+        + (f" (all of magnitude >= {t['decode_over_min_ref']:.3f}, where half a bf16 spacing "
+           f"is 1.56e-2)" if t["decode_over_abs_tol"] else "")
+        + f"; prefill: {t['over_abs_tol']} elements above 1e-2"
         + (f" (smallest |ref| {t['over_abs_tol_min_ref']:.3f}, largest error "
            f"{t['over_abs_tol_max_err']:.4e}): " + "; ".join(t["over_abs_tol_where"])
            if t["over_abs_tol"] else ""))

@@ -2,10 +2,12 @@
 
 Runs a further sweep of seeded random prefill cases and then looks at the running tally that
 helpers.assert_parity keeps for the whole process: after the other GPU tests that is the whole
-suite, alone it is this sweep.  Every decode comparison runs under the plain 1e-2 bound (an
-element above it fails its own test), so anything counted here is a prefill output that passed
-under the bound derived from the kernel's arithmetic; they must stay a handful among millions
-(most come from the two stress cases whose softmax is nearly one-hot: scale 8 and scale -0.25).
+suite, alone it is this sweep.  Every decode comparison runs under half a bf16 spacing plus
+5e-4, which is below 1e-2 wherever a bf16 output can be that close at all (|ref| < 4); the
+decode elements above 1e-2 must therefore all have magnitude 4 or more.  The prefill outputs
+that passed under the bound derived from the kernel's arithmetic must stay a handful among
+millions (most come from the two stress cases whose softmax is nearly one-hot: scale 8 and
+scale -0.25).
 """
 import pytest
 
@@ -23,3 +25,7 @@ def test_elements_above_the_plain_bound_are_rare_large_prefill_outputs():
     print(f"\nparity tally: {t['over_abs_tol']} of {t['amended_elements']} prefill elements above "
           f"1e-2 ({t['elements']} elements compared in all): {t['over_abs_tol_where']}")
     assert t["over_abs_tol"] <= 2 + 2e-5 * t["amended_elements"]
+    print(f"decode: {t['decode_over_abs_tol']} of {t['decode_elements']} elements above 1e-2, "
+          f"smallest magnitude {t['decode_over_min_ref']}")
+    assert t["decode_over_min_ref"] >= 4.0
+    assert t["decode_over_abs_tol"] <= 2 + 1e-6 * t["decode_elements"]
