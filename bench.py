@@ -196,8 +196,8 @@ def config_of(spec, world: int = 1, parallelism: str = ""):
 # captures summarised under profiles/, keyed by (workload, context tokens, H, Hkv, D, partition
 # size the plan chose).  Any other size, shape or partition size has no capture: null.
 NCU_TRAFFIC = {
-    ("cfg3_fullpool_mixed_gqa", 383921, 32, 8, 128, 512): 1596370816,
-    ("cfg2_llama2_7b_mha", 66297, 32, 32, 128, 256): 1100236416,
+    ("cfg3_fullpool_mixed_gqa", 383921, 32, 8, 128, 512): 1597484800,
+    ("cfg2_llama2_7b_mha", 66297, 32, 32, 128, 256): 1100038912,
 }
 
 

@@ -79,7 +79,7 @@ def test_ncu_traffic_is_reported_only_for_the_captured_shape_and_partition_size(
     from paper_2602_07878_b200 import workloads as wl
 
     spec = wl.config_spec(3)
-    assert bench.ncu_traffic(spec, 512) == 1596370816
+    assert bench.ncu_traffic(spec, 512) == 1597484800
     assert bench.ncu_traffic(spec, 256) is None
     assert bench.ncu_traffic(wl.config_spec(3, scale_down=8), 512) is None   # same name, smaller
     other = wl.make_spec(spec.name, seq_lens=spec.seq_lens, num_q_heads=16, num_kv_heads=8,
