@@ -108,12 +108,20 @@ int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch, int64_t max_tot
  *   k_cache      dev bf16, one layer, laid out per `shape`; v_cache likewise
  *   block_tables dev int32 [batch, max_blocks_per_seq] row-major; entries at or beyond
  *                ceil(seq_lens[b] / block_size) are never read
- *   seq_lens     dev int32 [batch]; 0 gives a row of zeros
+ *   seq_lens     dev int32 [batch]; 0 gives a row of zeros.  The plan kernel reads them while
+ *                the kernel before it in the stream may still run, if that kernel releases
+ *                its dependents early (programmatic dependent launch; the combine kernel of
+ *                the previous pa_decode call does, no kernel of this library writes
+ *                seq_lens).  Copies, memsets and kernels that do not release their dependents
+ *                early are complete before it reads, as stream order says.
  *   scale        softmax scale (e.g. 1/sqrt(D))
  *   out          dev bf16 [batch, H, D], contiguous, 16-byte aligned
  *   workspace    dev, >= pa_workspace_bytes(...), 256-byte aligned; contents are scratch.
  *                One call at a time per workspace: calls that may overlap on the GPU (different
- *                streams) need a workspace each
+ *                streams) need a workspace each.  Do not hand the same buffer to pa_prefill /
+ *                pa_prefill_split as their workspace: consecutive calls of the library on
+ *                one stream overlap at their edges, and only pa_decode calls among themselves
+ *                keep out of each other's way inside a shared workspace
  *   partition_tokens  0 = choose per call from the batch's total length; otherwise a
  *                multiple of 16 in [16, 512]: sequences longer than this are split into
  *                partitions of this many tokens that run in parallel and are merged by
@@ -125,6 +133,8 @@ int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch, int64_t max_tot
  *                the GPU never reads outside the pool.
  * Slots of the last block beyond seq_lens[b] may hold anything (NaN included).
  * Three kernels are enqueued (plan, partition attention, combine); nothing is synced.
+ * The workspace holds two plan regions used in turn, so the plan kernel of a call runs beside
+ * the combine kernel of the call before it on the same stream and workspace.
  */
 int pa_decode(const pa_shape* shape, const void* q, const void* k_cache, const void* v_cache,
               const int32_t* block_tables, int32_t max_blocks_per_seq, const int32_t* seq_lens,

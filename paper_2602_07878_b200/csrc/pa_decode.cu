@@ -13,6 +13,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -30,7 +31,9 @@ namespace pk {
 // ======================================================================================
 // plan kernel (one CTA): validate lengths, pick the partition size, list the work items
 // ======================================================================================
-constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_THREADS = 256;   // small enough to sit beside the previous call's combine CTAs
+constexpr int PLAN_WARPS = PLAN_THREADS / 32;
+constexpr int SEQ_CACHE = 1024;     // sequences whose (length, first partial) stay in shared memory
 
 constexpr int COMBINE_LONG = 32;  // rows with more partitions get a whole CTA in the combine
 
@@ -44,12 +47,11 @@ struct PlanParams {
     int no_direct;      // 1 = every sequence goes through the combine kernel
     int64_t item_cap;   // records the workspace can hold
     int total_warps;    // decode warps on the chip
-    int* hdr;
-    int2* seq_info;     // per sequence: (first partial index, partitions)
-    // the sequences whose rows the combine kernel writes: those with more than COMBINE_LONG
-    // partitions from the front, those with 0 or 2..COMBINE_LONG partitions from the back
-    int* multi;
-    int4* records;      // per item: (b, tok0, ntok | flags, partial index)
+    // Of the region this call fills: seq_info holds per sequence (first partial index,
+    // partitions); multi lists the sequences whose rows the combine kernel writes, those with
+    // more than COMBINE_LONG partitions from the front, those with 0 or 2..COMBINE_LONG from the
+    // back; records holds per item (b, tok0, ntok | flags, partial index).
+    PlanAddr plan;
     int* status;
 };
 
@@ -61,29 +63,36 @@ __device__ __forceinline__ int clamp_len(int L, int max_tok, bool& bad) {
     return L;
 }
 
-__global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanParams p) {
+// The kernel reads seq_lens and fills the plan region that the previous call on this workspace
+// did not use, and only then waits for the kernels before it in the stream: launched behind
+// the combine kernel of the previous call, it runs beside it.  (What precedes it in the stream
+// and lets its dependents go early must therefore not be what writes seq_lens; no kernel of
+// this library does.)
+__global__ void __launch_bounds__(PLAN_THREADS) pa_plan_kernel(const PlanParams p) {
     // per warp: items for each candidate size, items of the forced size, then for each candidate
     // the items of sequences that are split (their rows go through the combine) and the tokens
-    __shared__ long long red[10][32];
+    __shared__ long long red[10][PLAN_WARPS];
     __shared__ int s_P, s_bad;
     __shared__ int hist[MAX_PART / BS + 1], start[MAX_PART / BS + 1], cursor[MAX_PART / BS + 1];
-    __shared__ int scan_warp[32];
+    __shared__ int scan_warp[PLAN_WARPS];
     __shared__ int s_carry, s_multi, s_long;
-    // (length, first partial index) of the first PLAN_THREADS sequences: pass 3 reads them here
-    // instead of loading back what pass 2 has just written to global memory
-    __shared__ int2 s_seq[PLAN_THREADS];
+    __shared__ int2 s_seq[SEQ_CACHE];  // (length, first partial index) of the first sequences
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int max_tok = p.max_blocks * BS;
     const int cand[4] = {64, 128, 256, 512};
     pdl_launch_dependents();  // the attention kernel may set up while the plan is made
-    pdl_wait();               // the workspace may still be in use by the previous call
+    // The switch was last written at the end of an earlier call's plan kernel, and that call's
+    // attention kernel has started since: no wait is needed to read it.
+    const int gen = p.plan.fixed[HDR_GEN] + 1;
+    const PlanView pv = plan_view(p.plan, gen);
 
     // ---- pass 1: item counts for each candidate partition size ------------------------
     long long cnt[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     bool bad = false;
     for (int b = tid; b < p.batch; b += PLAN_THREADS) {
         const int L = clamp_len(p.seq_lens[b], max_tok, bad);
+        if (b < SEQ_CACHE) s_seq[b].x = L;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const int np = (L + cand[c] - 1) / cand[c];
@@ -109,7 +118,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
         long long tot[10];
 #pragma unroll
         for (int c = 0; c < 10; ++c) {
-            long long v = red[c][lane];
+            long long v = lane < PLAN_WARPS ? red[c][lane] : 0;
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
             tot[c] = v;
         }
@@ -142,109 +151,130 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) pa_plan_kernel(const PlanPara
     }
     __syncthreads();
     const int P = s_P;
+    int n_items = 0;
     if (P == 0) {  // plan does not fit: no work, combine writes zero rows
         for (int b = tid; b < p.batch; b += PLAN_THREADS) {
-            p.seq_info[b] = make_int2(0, 0);
-            p.multi[b] = b;
+            pv.seq_info[b] = make_int2(0, 0);
+            pv.multi[b] = b;
         }
         if (tid == 0) {
-            p.hdr[HDR_N_MULTI] = p.batch;
-            p.hdr[HDR_N_LONG] = 0;
-            p.hdr[HDR_N_ITEMS] = 0;
-            p.hdr[HDR_N_UNITS] = 0;
-            p.hdr[HDR_P] = 0;
-            p.hdr[HDR_COUNTER] = 3 * p.total_warps;
+            pv.hdr[HDR_N_MULTI] = p.batch;
+            pv.hdr[HDR_N_LONG] = 0;
+            pv.hdr[HDR_N_ITEMS] = 0;
+            pv.hdr[HDR_N_UNITS] = 0;
+            pv.hdr[HDR_P] = 0;
+            pv.hdr[HDR_COUNTER] = 3 * p.total_warps;
             atomicOr(p.status, PA_STATUS_WORKSPACE | (s_bad ? PA_STATUS_BAD_SEQ_LEN : 0));
         }
-        return;
-    }
-
-    // ---- pass 2: exclusive scan of partitions per sequence, histogram of item sizes ----
-    const int full_bin = P / BS;
-    for (int base = 0; base < p.batch; base += PLAN_THREADS) {
-        const int b = base + tid;
-        int np = 0;
-        if (b < p.batch) {
-            bool dummy = false;
-            const int L = clamp_len(p.seq_lens[b], max_tok, dummy);
-            np = (L + P - 1) / P;
-            // merged (or zeroed) by the combine kernel
-            if (np > COMBINE_LONG) p.multi[atomicAdd(&s_long, 1)] = b;
-            else if (np != 1) p.multi[p.batch - 1 - atomicAdd(&s_multi, 1)] = b;
-            if (np > 0) {
-                if (np > 1) atomicAdd(&hist[full_bin], np - 1);
-                const int last = L - (np - 1) * P;
-                atomicAdd(&hist[(last + BS - 1) / BS], 1);
-            }
-        }
-        int incl = np;
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) scan_warp[warp] = incl;
-        __syncthreads();
-        if (warp == 0) {
-            int v = scan_warp[lane];
-            for (int o = 1; o < 32; o <<= 1) {
-                const int u = __shfl_up_sync(0xffffffffu, v, o);
-                if (lane >= o) v += u;
-            }
-            scan_warp[lane] = v;  // inclusive over warps
-        }
-        __syncthreads();
-        const int warp_off = warp == 0 ? 0 : scan_warp[warp - 1];
-        const int carry = s_carry;
-        if (b < p.batch) {
-            const int first = carry + warp_off + incl - np;
-            p.seq_info[b] = make_int2(first, np);
-            if (base == 0) {
+    } else {
+        // ---- pass 2: exclusive scan of partitions per sequence, histogram of item sizes ----
+        const int full_bin = P / BS;
+        for (int base = 0; base < p.batch; base += PLAN_THREADS) {
+            const int b = base + tid;
+            int np = 0;
+            if (b < p.batch) {
                 bool dummy = false;
-                s_seq[tid] = make_int2(clamp_len(p.seq_lens[b], max_tok, dummy), first);
+                const int L = b < SEQ_CACHE ? s_seq[b].x : clamp_len(p.seq_lens[b], max_tok, dummy);
+                np = (L + P - 1) / P;
+                // merged (or zeroed) by the combine kernel
+                if (np > COMBINE_LONG) pv.multi[atomicAdd(&s_long, 1)] = b;
+                else if (np != 1) pv.multi[p.batch - 1 - atomicAdd(&s_multi, 1)] = b;
+                if (np > 0) {
+                    if (np > 1) atomicAdd(&hist[full_bin], np - 1);
+                    const int last = L - (np - 1) * P;
+                    atomicAdd(&hist[(last + BS - 1) / BS], 1);
+                }
             }
+            int incl = np;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) scan_warp[warp] = incl;
+            __syncthreads();
+            // inclusive over warps, every warp for itself
+            int upto = 0, total = 0;
+#pragma unroll
+            for (int w = 0; w < PLAN_WARPS; ++w) {
+                const int v = scan_warp[w];
+                if (w < warp) upto += v;
+                total += v;
+            }
+            const int carry = s_carry;
+            if (b < p.batch) {
+                const int first = carry + upto + incl - np;
+                pv.seq_info[b] = make_int2(first, np);
+                if (b < SEQ_CACHE) s_seq[b].y = first;
+            }
+            __syncthreads();
+            if (tid == 0) s_carry = carry + total;
         }
         __syncthreads();
-        if (tid == 0) s_carry = carry + scan_warp[31];
-        __syncthreads();
-    }
-    const int n_items = s_carry;
-    if (warp == 0) {  // larger items first: exclusive scan of the histogram from the top bin down
-        static_assert(MAX_PART / BS == 32, "one lane per bin");
-        const int nb = MAX_PART / BS - lane;
-        const int v = hist[nb];
-        int incl = v;
-        for (int o = 1; o < 32; o <<= 1) {
-            const int u = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += u;
+        n_items = s_carry;
+        if (warp == 0) {  // larger items first: exclusive scan of the histogram from the top bin down
+            static_assert(MAX_PART / BS == 32, "one lane per bin");
+            const int nb = MAX_PART / BS - lane;
+            const int v = hist[nb];
+            int incl = v;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += u;
+            }
+            start[nb] = incl - v;
         }
-        start[nb] = incl - v;
-    }
-    if (tid == 0) {
-        p.hdr[HDR_N_ITEMS] = n_items;
-        p.hdr[HDR_N_MULTI] = s_multi;
-        p.hdr[HDR_N_LONG] = s_long;
-        p.hdr[HDR_N_UNITS] = n_items * p.Hkv;
-        p.hdr[HDR_P] = P;
-        p.hdr[HDR_COUNTER] = 3 * p.total_warps;
-        if (s_bad) atomicOr(p.status, PA_STATUS_BAD_SEQ_LEN);
-    }
-    __syncthreads();
+        if (tid == 0) {
+            pv.hdr[HDR_N_ITEMS] = n_items;
+            pv.hdr[HDR_N_MULTI] = s_multi;
+            pv.hdr[HDR_N_LONG] = s_long;
+            pv.hdr[HDR_N_UNITS] = n_items * p.Hkv;
+            pv.hdr[HDR_P] = P;
+            pv.hdr[HDR_COUNTER] = 3 * p.total_warps;
+            if (s_bad) atomicOr(p.status, PA_STATUS_BAD_SEQ_LEN);
+        }
+        __syncthreads();
 
-    // ---- pass 3: one warp per sequence, lanes over its partitions ------------------------
-    for (int b = warp; b < p.batch; b += PLAN_THREADS / 32) {
-        bool dummy = false;
-        const int L = b < PLAN_THREADS ? s_seq[b].x : clamp_len(p.seq_lens[b], max_tok, dummy);
-        const int np = (L + P - 1) / P;
-        if (np == 0) continue;
-        const int first = b < PLAN_THREADS ? s_seq[b].y : p.seq_info[b].x;
-        for (int part = lane; part < np; part += 32) {
+        // ---- pass 3: the records, larger items first ------------------------------------------
+        auto emit = [&](int b, int L, int np, int first, int part) {
             const int tok0 = part * P;
             const int ntok = min(P, L - tok0);
             const int nb = (ntok + BS - 1) / BS;
             const int pos = start[nb] + atomicAdd(&cursor[nb], 1);
-            p.records[pos] =
+            pv.records[pos] =
                 make_int4(b, tok0, ntok | (np == 1 && !p.no_direct ? REC_DIRECT : 0), first + part);
+        };
+        if (p.batch <= SEQ_CACHE) {
+            // one thread per item: its sequence is the last one whose first partial index is not
+            // above the item (sequences without tokens share theirs with the next one)
+            for (int j = tid; j < n_items; j += PLAN_THREADS) {
+                int lo = 0, hi = p.batch - 1;
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (s_seq[mid].y <= j) lo = mid;
+                    else hi = mid - 1;
+                }
+                const int2 sq = s_seq[lo];
+                emit(lo, sq.x, (sq.x + P - 1) / P, sq.y, j - sq.y);
+            }
+        } else {
+            // one warp per sequence, lanes over its partitions
+            for (int b = warp; b < p.batch; b += PLAN_WARPS) {
+                bool dummy = false;
+                const int L = b < SEQ_CACHE ? s_seq[b].x : clamp_len(p.seq_lens[b], max_tok, dummy);
+                const int np = (L + P - 1) / P;
+                if (np == 0) continue;
+                const int first = b < SEQ_CACHE ? s_seq[b].y : pv.seq_info[b].x;
+                for (int part = lane; part < np; part += 32) emit(b, L, np, first, part);
+            }
         }
+    }
+    // Everything above went to a region that no kernel in flight reads.  This grid must not
+    // complete before the kernels of the previous call have (the attention kernel behind it
+    // waits for this grid only), and the switch must not move while they may still read it.
+    pdl_wait();
+    if (tid == 0) {
+        p.plan.fixed[HDR_GEN] = gen;
+        p.plan.fixed[HDR_N_ITEMS] = n_items;
+        p.plan.fixed[HDR_P] = P;
     }
 }
 
@@ -255,8 +285,7 @@ struct DecodeParams {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
     const int32_t* block_tables;
-    const int4* records;
-    int* hdr;
+    PlanAddr plan;
     float* partial_o;    // [item][H][D]  un-normalised
     float2* partial_ml;  // [item][H]     (running max in log2 units, row sum)
     int* status;
@@ -326,7 +355,8 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
     // theirs to read even before they wait for this grid's partial results.
     pdl_launch_dependents();
 
-    const int n_units = p.hdr[HDR_N_UNITS];
+    const PlanView pv = plan_view(p.plan, p.plan.fixed[HDR_GEN]);
+    const int n_units = pv.hdr[HDR_N_UNITS];
     const int total_warps = NW * gridDim.x;
     const int gw = warp * gridDim.x + blockIdx.x;
     const int G = p.G, H = p.H, Hkv = p.Hkv;
@@ -340,7 +370,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         if (valid) {
             const int item = w / Hkv;
             kvh = w - item * Hkv;
-            rec = __ldg(&p.records[item]);
+            rec = __ldg(&pv.records[item]);
         }
     };
     auto st_stash = [&](int ks, int i, uint32_t v) {
@@ -426,7 +456,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         load_record(gw, r0, k0, v0);
         load_record(gw + total_warps, r1, k1, v1);
         load_record(gw + 2 * total_warps, recB, kvhB, validB);
-        if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
+        if (lane == 0) wraw = atomicAdd(&pv.hdr[HDR_COUNTER], 1);
         build(r0, k0, v0, U0, false);
         if (QH) unpark_host(U0);
         build(r1, k1, v1, U1, true);
@@ -555,7 +585,7 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
             build(recB, kvhB, validB, U1, true);
             const int w = __shfl_sync(0xffffffffu, wraw, 0);
             load_record(w, recB, kvhB, validB);
-            if (lane == 0) wraw = atomicAdd(&p.hdr[HDR_COUNTER], 1);
+            if (lane == 0) wraw = atomicAdd(&pv.hdr[HDR_COUNTER], 1);
             if (iu == 1) iu = 0; else ib = 0;  // the issue cursor stays where it was
             cb = 0;
             A.reset();
@@ -567,12 +597,10 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
 // combine: one CTA per (sequence, query head)
 // ======================================================================================
 struct CombineParams {
-    const int2* seq_info;
-    const int* multi;  // pa_combine_rows_kernel: the sequences to write
+    PlanAddr plan;     // unused by COMBINE_MERGE
     const float* partial_o;
     const float2* partial_ml;
     __nv_bfloat16* out;
-    int* hdr;
     int rows;  // batch * H
     int H;
     int64_t out_stride;  // elements between the [H, D] output rows of consecutive sequences
@@ -600,9 +628,13 @@ __global__ void __launch_bounds__(128) pa_combine_kernel(const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     pdl_wait();  // partial results of the attention kernel are complete and visible
-    if (MODE != COMBINE_MERGE && row == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
     const int b = row / p.H, h = row - b * p.H;
-    const int2 info = MODE == COMBINE_MERGE ? make_int2(0, p.n_parts) : p.seq_info[b];
+    int2 info = make_int2(0, p.n_parts);
+    if (MODE != COMBINE_MERGE) {
+        const PlanView pv = plan_view(p.plan, p.plan.fixed[HDR_GEN]);
+        if (row == 0 && threadIdx.x == 0) pv.hdr[HDR_COUNTER] = p.counter_reset;
+        info = pv.seq_info[b];
+    }
     if (MODE == COMBINE_FINAL && info.y == 1) return;  // written directly by the attention kernel
     __nv_bfloat16* dst = p.out + (size_t)b * p.out_stride + (size_t)h * D;
     if (info.y == 0) {  // no tokens: a row of zeros (as a partial: weight zero)
@@ -754,16 +786,20 @@ int make_cache_map(CUtensorMap* map, const void* base, const pa_shape* s) {
 WsLayout ws_layout(int H, int D, int64_t batch, int64_t item_cap, size_t bytes) {
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
     WsLayout w;
+    w.off_region = up(HDR_WORDS * sizeof(int));
     w.off_seqinfo = up(HDR_WORDS * sizeof(int));
     w.off_multi = w.off_seqinfo + up((size_t)batch * sizeof(int2));
     w.off_records = w.off_multi + up((size_t)batch * sizeof(int));
-    const size_t per_item = sizeof(int4) + (size_t)H * sizeof(float2) + (size_t)H * D * sizeof(float);
+    // an item: its record in either plan region, its (max, sum) pairs and accumulator rows
+    const size_t per_item =
+        2 * sizeof(int4) + (size_t)H * sizeof(float2) + (size_t)H * D * sizeof(float);
     if (bytes > 0) {
-        const size_t fixed = w.off_records + 3 * 256;
+        const size_t fixed = w.off_region + 2 * w.off_records + 4 * 256;
         item_cap = bytes > fixed ? (int64_t)((bytes - fixed) / per_item) : 0;
     }
     w.item_cap = item_cap;
-    w.off_ml = w.off_records + up((size_t)item_cap * sizeof(int4));
+    w.region_bytes = w.off_records + up((size_t)item_cap * sizeof(int4));
+    w.off_ml = w.off_region + 2 * w.region_bytes;
     w.off_o = w.off_ml + up((size_t)item_cap * H * sizeof(float2));
     w.total = w.off_o + up((size_t)item_cap * H * D * sizeof(float));
     return w;
@@ -923,7 +959,7 @@ extern "C" int pa_workspace_bytes(const pa_shape* shape, int32_t max_batch,
     const int64_t pw = partition_tokens ? partition_tokens : 256;
     const int64_t cap = max_total_tokens / pw + max_batch + 1;
     WsLayout w = ws_layout(shape->num_q_heads, shape->head_dim, max_batch, cap, 0);
-    *bytes = w.total + 3 * 256;
+    *bytes = w.total + 4 * 256;
     return PA_OK;
 }
 
@@ -945,19 +981,20 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
     // its dependents go only after it has seen the plan), so the chain header -> list entry ->
     // sequence record of this CTA's first rows is walked while the attention kernel still runs.
     const int batch = p.rows / p.H;
-    const int n_long = p.hdr[HDR_N_LONG] * p.H, n_short = p.hdr[HDR_N_MULTI] * p.H;
+    const PlanView pv = plan_view(p.plan, p.plan.fixed[HDR_GEN]);
+    const int n_long = pv.hdr[HDR_N_LONG] * p.H, n_short = pv.hdr[HDR_N_MULTI] * p.H;
     int2 first_long = make_int2(0, 0), first_short = make_int2(0, 0);
     int first_long_b = 0, first_short_b = 0;
     if ((int)blockIdx.x < n_long) {
-        first_long_b = __ldg(&p.multi[blockIdx.x / p.H]);
-        first_long = p.seq_info[first_long_b];
+        first_long_b = __ldg(&pv.multi[blockIdx.x / p.H]);
+        first_long = pv.seq_info[first_long_b];
     }
     if ((int)blockIdx.x * 8 + warp < n_short) {
-        first_short_b = __ldg(&p.multi[batch - 1 - (blockIdx.x * 8 + warp) / p.H]);
-        first_short = p.seq_info[first_short_b];
+        first_short_b = __ldg(&pv.multi[batch - 1 - (blockIdx.x * 8 + warp) / p.H]);
+        first_short = pv.seq_info[first_short_b];
     }
     pdl_wait();  // partial results of the attention kernel are complete and visible
-    if (blockIdx.x == 0 && threadIdx.x == 0) p.hdr[HDR_COUNTER] = p.counter_reset;
+    if (blockIdx.x == 0 && threadIdx.x == 0) pv.hdr[HDR_COUNTER] = p.counter_reset;
 
     // sum of w_i * (o_i, l_i) over partitions i = start, start + stride, ... < np of one row
     auto gather = [&](int first, int np, int h, int start, int stride, float M, float (&acc)[VPL],
@@ -1021,8 +1058,8 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
     // ---- long rows: one per CTA ----
     for (int task = blockIdx.x; task < n_long; task += gridDim.x) {
         const bool first = task == (int)blockIdx.x;
-        const int b = first ? first_long_b : __ldg(&p.multi[task / p.H]), h = task % p.H;
-        const int2 info = first ? first_long : p.seq_info[b];
+        const int b = first ? first_long_b : __ldg(&pv.multi[task / p.H]), h = task % p.H;
+        const int2 info = first ? first_long : pv.seq_info[b];
         bool bad;
         const float M = row_max(info.x, info.y, h, bad);
         float acc[VPL];
@@ -1055,8 +1092,8 @@ __global__ void __launch_bounds__(256) pa_combine_rows_kernel(const __grid_const
     // ---- short rows: one per warp ----
     for (int task = blockIdx.x * 8 + warp; task < n_short; task += gridDim.x * 8) {
         const bool first = task == (int)blockIdx.x * 8 + warp;
-        const int b = first ? first_short_b : __ldg(&p.multi[batch - 1 - task / p.H]), h = task % p.H;
-        const int2 info = first ? first_short : p.seq_info[b];
+        const int b = first ? first_short_b : __ldg(&pv.multi[batch - 1 - task / p.H]), h = task % p.H;
+        const int2 info = first ? first_short : pv.seq_info[b];
         bool bad;
         const float M = row_max(info.x, info.y, h, bad);
         float acc[VPL];
@@ -1077,6 +1114,25 @@ static cudaError_t launch_combine(int D, int grid, cudaStream_t st, const Combin
     return D == 256   ? launch_pdl(pa_combine_kernel<256, MODE>, dim3(grid), dim3(128), 0, st, cp)
            : D == 128 ? launch_pdl(pa_combine_kernel<128, MODE>, dim3(grid), dim3(128), 0, st, cp)
                       : launch_pdl(pa_combine_kernel<64, MODE>, dim3(grid), dim3(128), 0, st, cp);
+}
+
+// CTAs of pa_combine_rows_kernel that one SM holds (asked once per head_dim).
+static int combine_rows_per_sm(int D, int* out) {
+    static std::mutex mu;
+    static int cached[3] = {0, 0, 0};
+    const int i = D == 64 ? 0 : D == 128 ? 1 : 2;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!cached[i]) {
+        int n = 0;
+        cudaError_t e =
+            D == 256   ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pa_combine_rows_kernel<256>, 256, 0)
+            : D == 128 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pa_combine_rows_kernel<128>, 256, 0)
+                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pa_combine_rows_kernel<64>, 256, 0);
+        if (e != cudaSuccess) return check_cuda(e);
+        cached[i] = n > 0 ? n : 1;
+    }
+    *out = cached[i];
+    return PA_OK;
 }
 
 // The three launches of a decode call.  `part` == nullptr: bf16 rows in `out`; otherwise one
@@ -1133,8 +1189,14 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     dp.q = static_cast<const __nv_bfloat16*>(q);
     dp.out = static_cast<__nv_bfloat16*>(out);
     dp.block_tables = block_tables;
-    dp.records = reinterpret_cast<const int4*>(ws + w.off_records);
-    dp.hdr = hdr;
+    PlanAddr pa;
+    pa.fixed = hdr;
+    pa.region0 = ws + w.off_region;
+    pa.region_bytes = w.region_bytes;
+    pa.off_seqinfo = w.off_seqinfo;
+    pa.off_multi = w.off_multi;
+    pa.off_records = w.off_records;
+    dp.plan = pa;
     dp.partial_o = reinterpret_cast<float*>(ws + w.off_o);
     dp.partial_ml = reinterpret_cast<float2*>(ws + w.off_ml);
     dp.status = status;
@@ -1165,10 +1227,7 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
         pp.no_direct = part != nullptr;
         pp.item_cap = w.item_cap;
         pp.total_warps = total_warps;
-        pp.hdr = hdr;
-        pp.seq_info = reinterpret_cast<int2*>(ws + w.off_seqinfo);
-        pp.multi = reinterpret_cast<int*>(ws + w.off_multi);
-        pp.records = reinterpret_cast<int4*>(ws + w.off_records);
+        pp.plan = pa;
         pp.status = status;
         count_launch();
         rc = check_cuda(launch_pdl(pa_plan_kernel, dim3(1), dim3(PLAN_THREADS), 0, st, pp));
@@ -1181,12 +1240,10 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     if (prof) cudaEventRecord(prof_ev.ev[2], st);
 
     CombineParams cp = {};
-    cp.seq_info = reinterpret_cast<const int2*>(ws + w.off_seqinfo);
-    cp.multi = reinterpret_cast<const int*>(ws + w.off_multi);
+    cp.plan = pa;
     cp.partial_o = dp.partial_o;
     cp.partial_ml = dp.partial_ml;
     cp.out = dp.out;
-    cp.hdr = hdr;
     cp.rows = batch * H;
     cp.H = H;
     cp.out_stride = out_stride;
@@ -1197,7 +1254,13 @@ static int decode_impl(const pa_shape* shape, const void* q, const void* k_cache
     }
     const int cgrid = cp.rows;
     count_launch();
-    const dim3 rgrid(8 * dev.sm_count), rblock(256);  // every SM full of warps with loads in flight
+    // One CTA fewer than the chip holds at once: the whole grid is resident together, so the
+    // next call's plan kernel is launched as soon as this grid has started, and one SM keeps
+    // threads and registers free for it.
+    int per_sm = 0;
+    rc = combine_rows_per_sm(D, &per_sm);
+    if (rc) return rc;
+    const dim3 rgrid(std::max(1, per_sm * dev.sm_count - 1)), rblock(256);
     rc = check_cuda(part       ? launch_combine<COMBINE_TO_PARTIAL>(D, cgrid, st, cp)
                     : D == 256 ? launch_pdl(pa_combine_rows_kernel<256>, rgrid, rblock, 0, st, cp)
                     : D == 128 ? launch_pdl(pa_combine_rows_kernel<128>, rgrid, rblock, 0, st, cp)

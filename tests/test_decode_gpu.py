@@ -197,6 +197,53 @@ def test_reuse_plan_flag_and_other_stream():
             assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
+def test_back_to_back_calls_with_different_plans_share_a_workspace():
+    """The plan kernel of a call runs beside the combine kernel of the call before it and fills
+    the plan region that call does not use.  Calls with different length sets (so different
+    work lists, partition counts and combine lists) are queued on one stream and one workspace
+    with no synchronisation in between; every call's rows must be the ones it gives alone."""
+    spec = wl.config_spec(3, scale_down=8)
+    q, k, v = small_inputs(spec)
+    g = GpuDecode(spec, q, k, v)
+    rng = np.random.default_rng(11)
+    base = spec.seq_lens.astype(np.int64)
+    variants = []
+    for i in range(5):
+        lens = base.copy()
+        pick = rng.random(lens.size)
+        lens[pick < 0.3] = 0                                  # rows of zeros through the combine
+        lens[(pick >= 0.3) & (pick < 0.6)] //= int(rng.integers(2, 9))
+        if i == 3:
+            lens[:] = np.minimum(lens, 40)                    # every sequence a single partition
+        variants.append(lens.astype(np.int32))
+    alone = []
+    for lens in variants:
+        g.lens.copy_(torch.from_numpy(lens).cuda())
+        alone.append(g.run().clone())
+        assert int(g.status.item()) == 0
+    ref = oracle.pa_decode(q, k, v, spec.block_tables, variants[1], spec.scale)
+    assert_parity(torch_to_f64(alone[1]), ref, "variant 1 alone")
+
+    dev_lens = [torch.from_numpy(l).cuda() for l in variants]
+    outs = [torch.full_like(g.q, float("nan")) for _ in range(12)]
+    order = [0, 1, 2, 3, 4, 3, 1, 1, 0, 4, 2, 0]
+    torch.cuda.synchronize()
+    for out, which in zip(outs, order):
+        api.pa_decode(g.q, g.k, g.v, g.tables, dev_lens[which], spec.scale, out, g.ws,
+                      dev_status=g.status)
+    # a call that keeps the plan of the call before it, then one that plans again
+    again = torch.full_like(g.q, float("nan"))
+    api.pa_decode(g.q, g.k, g.v, g.tables, dev_lens[order[-1]], spec.scale, again, g.ws,
+                  dev_status=g.status, flags=api.PA_FLAG_REUSE_PLAN)
+    last = torch.full_like(g.q, float("nan"))
+    api.pa_decode(g.q, g.k, g.v, g.tables, dev_lens[2], spec.scale, last, g.ws, dev_status=g.status)
+    torch.cuda.synchronize()
+    assert int(g.status.item()) == 0
+    g.check_guards()
+    for out, which in zip(outs + [again, last], order + [order[-1], 2]):
+        assert torch.equal(out.view(torch.int16), alone[which].view(torch.int16)), which
+
+
 def test_workspace_too_small_for_plan_is_reported():
     spec = wl.make_spec("t", seq_lens=[4096] * 8, num_q_heads=8, num_kv_heads=8, head_dim=64,
                         occupancy=0.9, seed=35)
