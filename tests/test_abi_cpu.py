@@ -60,6 +60,18 @@ def test_workspace_bytes_grows_and_validates(L):
         assert L.pa_workspace_bytes(ctypes.byref(s), 1, 1, p, ctypes.byref(out)) == api.ERR["ARG"]
 
 
+def test_workspace_bytes_holds_two_plan_regions_and_the_partial_records(L):
+    # per work item: a 16-byte record in each of the two plan regions, H (max, sum) pairs and H
+    # fp32 rows of D; per sequence: 8 + 4 bytes in each region; a few 256-byte roundings on top
+    s = good_shape()
+    H, D = s.num_q_heads, s.head_dim
+    for batch, tokens, P in [(1, 16, 0), (256, 400000, 0), (256, 400000, 64), (3000, 90000, 512)]:
+        items = tokens // (P or 256) + batch + 1
+        need = items * (2 * 16 + H * 8 + H * D * 4) + 2 * batch * 12
+        got = api.pa_workspace_bytes(s, batch, tokens, P)
+        assert need <= got <= need + 16 * 256, (batch, tokens, P, need, got)
+
+
 @pytest.mark.parametrize("field,value", [("head_dim", 96), ("block_size", 32), ("num_q_heads", 30),
                                          ("num_q_heads", 8 * 17), ("dtype", 0),
                                          ("stride_tok", 132), ("num_blocks", 0),
