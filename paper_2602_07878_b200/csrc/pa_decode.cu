@@ -19,6 +19,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 #include <utility>
 #include <vector>
 
@@ -462,7 +463,10 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         build(r1, k1, v1, U1, true);
     }
 
-    AttnFrag<D, HI, true> A;
+    // groups of at most 8 heads at head_dim 256 take the operand-exchanged form: half the MMAs
+    // and half the accumulator registers, where a scheduler holds a single warp
+    constexpr bool TR = !HI && !QH && D == 256;
+    std::conditional_t<TR, AttnFragT<D, true>, AttnFrag<D, HI, true>> A;
     A.init_lane(lane);
     A.reset();
 
@@ -518,64 +522,102 @@ pa_decode_kernel(const __grid_constant__ CUtensorMap kmap,
         // ---- unit finished: write its result, move to the next unit -----------------------------
         if (cb == U0.nblk) {
             A.reduce_row_sums();
-            const float l0 = A.l0, l1 = A.l1, m0 = A.m0, m1 = A.m1;
-            auto& o = A.o;
-            const int h0 = U0.kvh * G + g;
-            if (QH && U0.direct) {
-                // host-resident tensors: the rows go out as whole 16-byte pieces per lane (512
-                // contiguous bytes per instruction) instead of 4-byte fragments
-                const float i0 = U0.bad ? 0.f : 1.f / l0;
+            if constexpr (TR) {
+                // this thread: heads 2t and 2t + 1 of the group, dims 16 jj + g and + 8
+                const int hA = U0.kvh * G + 2 * t;
+                const bool okA = 2 * t < G, okB = 2 * t + 1 < G;
+                if (U0.direct) {
+                    // neighbours in g exchange a value, so that each stores two dims of one head
+                    const float iA = U0.bad ? 0.f : 1.f / A.l0, iB = U0.bad ? 0.f : 1.f / A.l1;
+                    const bool even = (g & 1) == 0;
+                    const bool ok = even ? okA : okB;
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(
+                        p.out + (size_t)U0.b * p.out_stride + (size_t)(hA + (even ? 0 : 1)) * D);
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(qrows + (g * D + nt * 8 + 2 * t) * 2),
-                                 "r"(U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0))
-                                 : "memory");
-                __syncwarp();
-                uint4* orow = reinterpret_cast<uint4*>(p.out + (size_t)U0.b * p.out_stride +
-                                                       (size_t)U0.kvh * G * D);
+                    for (int jj = 0; jj < D / 16; ++jj) {
 #pragma unroll
-                for (int i = 0; i < D / 32; ++i) {
-                    const int piece = i * 32 + lane;
-                    if (piece / (D / 8) < G) {
-                        uint4 w;
-                        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
-                                     : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
-                                     : "r"(qrows + piece * 16));
-                        orow[piece] = w;
+                        for (int hf = 0; hf < 2; ++hf) {
+                            const float xA = A.o[jj][2 * hf] * iA, xB = A.o[jj][2 * hf + 1] * iB;
+                            const float got = __shfl_xor_sync(0xffffffffu, even ? xB : xA, 4);
+                            const uint32_t w = even ? pack_bf16x2(xA, got) : pack_bf16x2(got, xB);
+                            if (ok) dst[(16 * jj + 8 * hf + (g & ~1)) >> 1] = w;
+                        }
+                    }
+                } else {
+                    const float nanv = __int_as_float(0x7fc00000);
+                    const size_t rowA = (size_t)U0.pidx * H + hA;
+                    float* dA = p.partial_o + rowA * D;
+                    float* dB = dA + D;
+#pragma unroll
+                    for (int jj = 0; jj < D / 16; ++jj) {
+                        if (okA) dA[16 * jj + g] = A.o[jj][0], dA[16 * jj + g + 8] = A.o[jj][2];
+                        if (okB) dB[16 * jj + g] = A.o[jj][1], dB[16 * jj + g + 8] = A.o[jj][3];
+                    }
+                    if (g == 0) {
+                        if (okA) p.partial_ml[rowA] = make_float2(U0.bad ? nanv : A.m0, A.l0);
+                        if (okB) p.partial_ml[rowA + 1] = make_float2(U0.bad ? nanv : A.m1, A.l1);
                     }
                 }
-                __syncwarp();
-            } else if (U0.direct) {
-                const float i0 = U0.bad ? 0.f : 1.f / l0, i1 = U0.bad ? 0.f : 1.f / l1;
-                if (g < G) {
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(
-                        p.out + (size_t)U0.b * p.out_stride + (size_t)h0 * D);
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-                        dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0);
-                }
-                if (HI && g + 8 < G) {
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(
-                        p.out + (size_t)U0.b * p.out_stride + (size_t)(h0 + 8) * D);
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-                        dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][2] * i1, o[nt][3] * i1);
-                }
             } else {
-                const float nanv = __int_as_float(0x7fc00000);
-                if (g < G) {
-                    const size_t row = (size_t)U0.pidx * H + h0;
-                    float2* dst = reinterpret_cast<float2*>(p.partial_o + row * D);
+                const float l0 = A.l0, l1 = A.l1, m0 = A.m0, m1 = A.m1;
+                auto& o = A.o;
+                const int h0 = U0.kvh * G + g;
+                if (QH && U0.direct) {
+                    // host-resident tensors: the rows go out as whole 16-byte pieces per lane (512
+                    // contiguous bytes per instruction) instead of 4-byte fragments
+                    const float i0 = U0.bad ? 0.f : 1.f / l0;
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) dst[nt * 4 + t] = make_float2(o[nt][0], o[nt][1]);
-                    if (t == 0) p.partial_ml[row] = make_float2(U0.bad ? nanv : m0, l0);
-                }
-                if (HI && g + 8 < G) {
-                    const size_t row = (size_t)U0.pidx * H + h0 + 8;
-                    float2* dst = reinterpret_cast<float2*>(p.partial_o + row * D);
+                    for (int nt = 0; nt < NT; ++nt)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(qrows + (g * D + nt * 8 + 2 * t) * 2),
+                                     "r"(U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0))
+                                     : "memory");
+                    __syncwarp();
+                    uint4* orow = reinterpret_cast<uint4*>(p.out + (size_t)U0.b * p.out_stride +
+                                                           (size_t)U0.kvh * G * D);
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) dst[nt * 4 + t] = make_float2(o[nt][2], o[nt][3]);
-                    if (t == 0) p.partial_ml[row] = make_float2(U0.bad ? nanv : m1, l1);
+                    for (int i = 0; i < D / 32; ++i) {
+                        const int piece = i * 32 + lane;
+                        if (piece / (D / 8) < G) {
+                            uint4 w;
+                            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                                         : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                                         : "r"(qrows + piece * 16));
+                            orow[piece] = w;
+                        }
+                    }
+                    __syncwarp();
+                } else if (U0.direct) {
+                    const float i0 = U0.bad ? 0.f : 1.f / l0, i1 = U0.bad ? 0.f : 1.f / l1;
+                    if (g < G) {
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(
+                            p.out + (size_t)U0.b * p.out_stride + (size_t)h0 * D);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+                            dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][0] * i0, o[nt][1] * i0);
+                    }
+                    if (HI && g + 8 < G) {
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(
+                            p.out + (size_t)U0.b * p.out_stride + (size_t)(h0 + 8) * D);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+                            dst[nt * 4 + t] = U0.bad ? 0u : pack_bf16x2(o[nt][2] * i1, o[nt][3] * i1);
+                    }
+                } else {
+                    const float nanv = __int_as_float(0x7fc00000);
+                    if (g < G) {
+                        const size_t row = (size_t)U0.pidx * H + h0;
+                        float2* dst = reinterpret_cast<float2*>(p.partial_o + row * D);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) dst[nt * 4 + t] = make_float2(o[nt][0], o[nt][1]);
+                        if (t == 0) p.partial_ml[row] = make_float2(U0.bad ? nanv : m0, l0);
+                    }
+                    if (HI && g + 8 < G) {
+                        const size_t row = (size_t)U0.pidx * H + h0 + 8;
+                        float2* dst = reinterpret_cast<float2*>(p.partial_o + row * D);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) dst[nt * 4 + t] = make_float2(o[nt][2], o[nt][3]);
+                        if (t == 0) p.partial_ml[row] = make_float2(U0.bad ? nanv : m1, l1);
+                    }
                 }
             }
             // advance the fetch pipeline
