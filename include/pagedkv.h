@@ -293,8 +293,12 @@ int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const 
  * the recomputation chunk of Section 5.1.2 / Appendix B.1: a 512-token chunk of one long
  * victim yields fewer 128-row tiles than the GPU has SMs, while each tile walks tens of
  * thousands of cached tokens).  The result is the same function of the inputs as pa_prefill;
- * only the order of the fp32 sums differs.  A sequence whose context spans more than one
- * split leaves per-split partial rows in the workspace, merged by a third kernel.
+ * only the order of the fp32 sums differs.  The units of a sequence whose context spans more
+ * than one split leave per-split partial rows in the workspace and count themselves in; the
+ * unit of a row group that arrives last merges them into the output rows, in the same kernel.
+ * The counters carry the number of the call on that workspace (kept by the library, per
+ * workspace address), so nothing in the workspace needs to be cleared by the caller; the first
+ * call the library sees on a workspace enqueues one memset of its counters.
  *
  *   kv_split_tokens   0: the library chooses tile shape and split length from the chunk
  *                     size, max_blocks_per_seq (taken as the bound of every context: pass
@@ -306,8 +310,8 @@ int pa_prefill(const pa_shape* shape, const void* q, const void* k_cache, const 
  *                     used up to what pa_prefill_split_workspace_bytes(shape, batch, total_q,
  *                     splits) says fits.
  * pa_prefill is this call with kv_split_tokens = 0.
- * One to three kernels are enqueued (plan, attention, merge).  Errors as for pa_prefill; a split that met a bad
- * block id zeroes the rows that depend on it.
+ * One or two kernels are enqueued (plan, attention).  Errors as for pa_prefill; a split that met
+ * a bad block id zeroes the rows that depend on it.
  */
 int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t max_batch,
                                      int32_t max_total_q, int32_t max_splits, size_t* bytes);

@@ -342,17 +342,146 @@ struct PrefillTcParams {
     PrefillParams base;
     int tokens_per_tile;  // 128 / G, rounded down: rows tokens_per_tile * G .. 127 of a tile are idle
     // KV split: a unit covers `split_steps` 64-token steps of its tile's visible context (0 =
-    // all of it).  A sequence with more than one split leaves, per (query row, split), an
-    // un-normalised fp32 output row in part_o[(row * split_cap + s) * D] and its reference
-    // exponent and weight sum in part_ml[(row * split_cap + s) * 2]; row = query token * H +
-    // head.  A negative sum marks a split that met a bad block id.
+    // all of it).  The units of one row group (same query tokens, same KV head) each leave a
+    // partial record -- per row the reference exponent and weight sum (a negative sum marks a
+    // split that met a bad block id) and the un-normalised fp32 output row -- and count
+    // themselves in; the one that arrives last merges the records into the output rows.
+    // Records are laid out for threads that own a row each:
+    //   part_ml[((group * split_cap + split) * NT + tile) * 128 + row]              float2
+    //   part_o [(((group * split_cap + split) * NT + tile) * D/4 + chunk) * 128 + row]  float4
+    // group = ((q0 + tok0) / tokens per CTA + sequence) * Hkv + KV head.
     int split_steps, split_cap;
     float* part_ml;
     float* part_o;
+    // arrive[group]: (epoch << 8) | units arrived in the call numbered `epoch` on this
+    // workspace; a word from another call counts as zero, so nothing needs resetting
+    int* arrive;
+    int epoch;
     // Batches of at most 32 sequences need no plan kernel: every CTA validates the lengths and
     // scans the unit counts itself (one warp, a few hundred cycles) and only CTA 0 reports.
     int fold_plan, total_q;
 };
+
+// The merge of a row group by its last unit, two to four splits (the usual case):
+//   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s.
+template <int D, int NT>
+__device__ __forceinline__ void merge_few_splits(int n_vis, int split, float m_ref, float l,
+                                              bool bad_own, const float2* ml_all,
+                                              const float4* o_all, size_t rec0, int row,
+                                              bool row_ok, __nv_bfloat16* dst, uint32_t tcol,
+                                              uint32_t lane_base) {
+    using namespace tc;
+    // The last unit of the row group, two to four splits (the usual case):
+    //   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s.
+    // Its own row is still in tensor memory; the pairs of the other splits come in
+    // one round trip, their rows 32 floats at a time with the loads of two splits
+    // in flight together.
+    __threadfence();
+    float2 ml[4];
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {
+        ml[sp] = make_float2(-INFINITY, 0.f);
+        if (sp == split) ml[sp] = make_float2(m_ref, bad_own ? -1.f : l);
+        else if (sp < n_vis && row_ok)
+            ml[sp] = __ldcg(&ml_all[(rec0 + (size_t)sp * NT) * 128 + row]);
+    }
+    const float M = fmaxf(fmaxf(ml[0].x, ml[1].x), fmaxf(ml[2].x, ml[3].x));
+    const bool bad = ml[0].y < 0.f || ml[1].y < 0.f || ml[2].y < 0.f || ml[3].y < 0.f;
+    float w[4], lsum = 0.f;
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {
+        w[sp] = ml[sp].x == -INFINITY ? 0.f : ex2(ml[sp].x - M);
+        lsum = fmaf(w[sp], ml[sp].y, lsum);
+    }
+    const float inv = (bad || !(lsum > 0.f)) ? 0.f : 1.f / lsum;
+    float w_own = 0.f;
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {
+        w[sp] *= inv;
+        if (sp == split) w_own = w[sp];
+    }
+    // the other splits, in ascending order (at most three)
+    int oth[3] = {0, 0, 0};
+    {
+        int k = 0;
+#pragma unroll
+        for (int sp = 0; sp < 4; ++sp)
+            if (sp != split && sp < n_vis && k < 3) oth[k++] = sp;
+    }
+    const int n_oth = n_vis - 1;
+    auto w_of = [&](int sp) { return sp == 0 ? w[0] : sp == 1 ? w[1] : sp == 2 ? w[2] : w[3]; };
+#pragma unroll 1
+    for (int c = 0; c < D; c += 32) {
+        uint32_t o[32];
+        tmem_ld32(tcol + lane_base + 2 * STEP + c, o);
+        float4 x0[8], x1[8];
+        const float4* s0 = o_all + ((rec0 + (size_t)oth[0] * NT) * (D / 4) + (c >> 2)) * 128 + row;
+        const float4* s1 = o_all + ((rec0 + (size_t)oth[1] * NT) * (D / 4) + (c >> 2)) * 128 + row;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x0[i] = n_oth > 0 && row_ok ? __ldcg(s0 + (size_t)i * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x1[i] = n_oth > 1 && row_ok ? __ldcg(s1 + (size_t)i * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        tmem_wait_ld();
+        // The weighted rows are added in the order of their splits, whichever unit
+        // does the adding: the result does not depend on which one arrived last.
+        float acc[32];
+        const float wa = n_oth > 0 ? w_of(oth[0]) : 0.f, wb = n_oth > 1 ? w_of(oth[1]) : 0.f;
+        const bool own_first = split <= 1;  // this unit's row is among the first two terms
+        const float* xa = reinterpret_cast<const float*>(x0);
+        const float* xb = reinterpret_cast<const float*>(x1);
+        if (n_oth <= 2) {
+            // two or three splits: one fused chain in split order (the branch is
+            // the same for every thread of the CTA)
+            if (split == 0) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    acc[e] = fmaf(wb, xb[e], fmaf(wa, xa[e], w_own * __uint_as_float(o[e])));
+            } else if (split == 1) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    acc[e] = fmaf(wb, xb[e], fmaf(w_own, __uint_as_float(o[e]), wa * xa[e]));
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    acc[e] = fmaf(w_own, __uint_as_float(o[e]), fmaf(wb, xb[e], wa * xa[e]));
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                const float pa = w_own * __uint_as_float(o[e]);
+                const float pb = wa * xa[e], pc = wb * xb[e];
+                acc[e] = own_first ? (pa + pb) + pc : pb + pc;
+            }
+        }
+        if (n_oth > 2) {
+            const float4* s2 = o_all + ((rec0 + (size_t)oth[2] * NT) * (D / 4) + (c >> 2)) * 128 + row;
+            const float wc = w_of(oth[2]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 x = row_ok ? __ldcg(s2 + (size_t)i * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float xd[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float pa = w_own * __uint_as_float(o[4 * i + e]), pd = wc * xd[e];
+                    float& t = acc[4 * i + e];
+                    t = own_first ? t + pd : split == 2 ? (t + pa) + pd : (t + pd) + pa;
+                }
+            }
+        }
+        if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+                uint4 w4;
+                w4.x = bad ? 0u : pack_bf16x2(acc[i], acc[i + 1]);
+                w4.y = bad ? 0u : pack_bf16x2(acc[i + 2], acc[i + 3]);
+                w4.z = bad ? 0u : pack_bf16x2(acc[i + 4], acc[i + 5]);
+                w4.w = bad ? 0u : pack_bf16x2(acc[i + 6], acc[i + 7]);
+                *reinterpret_cast<uint4*>(dst + c + i) = w4;
+            }
+        }
+    }
+}
 
 template <int D, int NT>
 __global__ void __launch_bounds__(tc::Cfg<D, NT>::THREADS, 1)
@@ -375,7 +504,8 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     auto bar = [&](int i) { return sbase + OFF_BAR + 8 * i; };
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + OFF_MISC);
-    // misc[0] = TMEM base address, misc[1] = abort flag, misc[2] = bad block id seen
+    // misc[0] = TMEM base address, misc[1] = abort flag, misc[2] = bad block id seen,
+    // misc[3] = this unit is the last of its row group to arrive
 
     // Dependents (the merge kernel, the next call) start once every CTA here has passed the
     // wait, i.e. when all that precedes this call in the stream is complete: they may then read
@@ -437,6 +567,10 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     const int n_steps = min(pos_max / STEP + 1 - j0, n_split > 1 ? tp.split_steps : 0x7fffffff);
     if (n_steps <= 0) return;                           // the tile sees nothing of this split
     const int nblk_seq = (L + BS - 1) / BS;
+    // the row group's index among all row groups of the call (see PrefillTcParams), and the
+    // number of splits whose units exist for it: those that start at or before its last position
+    const int group = ((q0 + tok0) / (NT * tpt) + b) * Hkv + kvh;
+    const int n_vis = min(n_split, (pos_max / STEP + 1 + tp.split_steps - 1) / max(tp.split_steps, 1));
     const int rows_used = tpt * G;                      // < 128 when G does not divide 128
 
     if (tid == 0) {
@@ -778,24 +912,109 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
         }
         // ---- epilogue: O / l -> bf16 rows, or the unit's partial record when the KV is split ----
         if (ok) ok = wait(tb + T_PVDONE + ((n_steps - 1) & 1), ((n_steps - 1) >> 1) & 1);
-        if (ok && n_split > 1) {
-            tc_fence_after_sync();
-            const size_t rec =
-                ((size_t)(q0 + qtok) * H + (size_t)kvh * G + hd) * tp.split_cap + split;
-            if (row_ok)
-                *reinterpret_cast<float2*>(tp.part_ml + rec * 2) =
-                    make_float2(m_ref, misc[2] != 0 ? -1.f : l);
-            float* dst = tp.part_o + rec * D;
+        if (n_split > 1) {
+            const float2* ml_all = reinterpret_cast<const float2*>(tp.part_ml);
+            const float4* o_all = reinterpret_cast<const float4*>(tp.part_o);
+            const size_t rec0 = (size_t)group * tp.split_cap * NT + ti;   // record of split s: + s * NT
+            if (ok) {
+                tc_fence_after_sync();
+                const size_t rec = rec0 + (size_t)split * NT;
+                if (row_ok)
+                    reinterpret_cast<float2*>(tp.part_ml)[rec * 128 + row] =
+                        make_float2(m_ref, misc[2] != 0 ? -1.f : l);
+                float4* dst = reinterpret_cast<float4*>(tp.part_o) + rec * (D / 4) * 128 + row;
 #pragma unroll 1
-            for (int c = 0; c < D; c += 32) {
-                uint32_t o[32];
-                tmem_ld32(tcol + lane_base + 2 * STEP + c, o);
-                tmem_wait_ld();
-                if (row_ok) {
+                for (int c = 0; c < D; c += 64) {  // two tensor-memory loads in flight
+                    uint32_t o[2][32];
+                    tmem_ld32(tcol + lane_base + 2 * STEP + c, o[0]);
+                    tmem_ld32(tcol + lane_base + 2 * STEP + c + 32, o[1]);
+                    tmem_wait_ld();
+                    if (row_ok) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<uint4*>(dst + c + i) =
-                            make_uint4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4)
+                                dst[(size_t)((c + 32 * hf + i) >> 2) * 128] = make_float4(
+                                    __uint_as_float(o[hf][i]), __uint_as_float(o[hf][i + 1]),
+                                    __uint_as_float(o[hf][i + 2]), __uint_as_float(o[hf][i + 3]));
+                    }
+                }
+            }
+            // The softmax warps of the CTA meet (every one of them gets here: all waits are
+            // bounded); one thread counts the unit in, unless some warp gave up.
+            asm volatile("bar.sync 1, %0;" ::"r"(NT * 128) : "memory");
+            if (warp == 0 && lane == 0) {
+                uint32_t last = 0;
+                // what the CTA's threads wrote before the barrier is visible to the GPU before
+                // the count is (the fence is cumulative over the barrier)
+                __threadfence();
+                if (misc[1] == 0) {
+                    int cur = *reinterpret_cast<volatile int*>(tp.arrive + group), nxt;
+                    for (;;) {
+                        nxt = ((cur >> 8) == tp.epoch ? cur : (tp.epoch << 8)) + 1;
+                        const int prev = atomicCAS(tp.arrive + group, cur, nxt);
+                        if (prev == cur) break;
+                        cur = prev;
+                    }
+                    last = (nxt & 255) == n_vis;
+                }
+                misc[3] = last;
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(NT * 128) : "memory");
+            if (misc[3] != 0 && n_vis <= 4) {
+                merge_few_splits<D, NT>(
+                    n_vis, split, m_ref, l, misc[2] != 0, ml_all, o_all, rec0, row, row_ok,
+                    p.out + ((size_t)(q0 + qtok) * H + (size_t)kvh * G + hd) * D, tcol, lane_base);
+            } else if (misc[3] != 0 && row_ok) {
+                // more than four splits: every record from memory, this unit's own included
+                __threadfence();
+                __nv_bfloat16* dst =
+                    p.out + ((size_t)(q0 + qtok) * H + (size_t)kvh * G + hd) * D;
+                {
+                    float M = -INFINITY;
+                    bool bad = false;
+                    for (int sp = 0; sp < n_vis; ++sp) {
+                        const float2 v = __ldcg(&ml_all[(rec0 + (size_t)sp * NT) * 128 + row]);
+                        M = fmaxf(M, v.x);
+                        bad |= v.y < 0.f;
+                    }
+                    float lsum = 0.f;
+                    for (int sp = 0; sp < n_vis; ++sp) {
+                        const float2 v = __ldcg(&ml_all[(rec0 + (size_t)sp * NT) * 128 + row]);
+                        lsum = fmaf(v.x == -INFINITY ? 0.f : ex2(v.x - M), v.y, lsum);
+                    }
+                    const float inv = (bad || !(lsum > 0.f)) ? 0.f : 1.f / lsum;
+#pragma unroll 1
+                    for (int c4 = 0; c4 < D / 4; c4 += 8) {
+                        float acc[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+                        for (int sp = 0; sp < n_vis; ++sp) {
+                            const size_t rec = rec0 + (size_t)sp * NT;
+                            const float mx = __ldcg(&ml_all[rec * 128 + row]).x;
+                            const float w = mx == -INFINITY ? 0.f : ex2(mx - M) * inv;
+                            const float4* src = o_all + (rec * (D / 4) + c4) * 128 + row;
+                            float4 x[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) x[i] = __ldcg(src + (size_t)i * 128);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                acc[4 * i] = fmaf(w, x[i].x, acc[4 * i]);
+                                acc[4 * i + 1] = fmaf(w, x[i].y, acc[4 * i + 1]);
+                                acc[4 * i + 2] = fmaf(w, x[i].z, acc[4 * i + 2]);
+                                acc[4 * i + 3] = fmaf(w, x[i].w, acc[4 * i + 3]);
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+                            uint4 w4;
+                            w4.x = bad ? 0u : pack_bf16x2(acc[i], acc[i + 1]);
+                            w4.y = bad ? 0u : pack_bf16x2(acc[i + 2], acc[i + 3]);
+                            w4.z = bad ? 0u : pack_bf16x2(acc[i + 4], acc[i + 5]);
+                            w4.w = bad ? 0u : pack_bf16x2(acc[i + 6], acc[i + 7]);
+                            *reinterpret_cast<uint4*>(dst + c4 * 4 + i) = w4;
+                        }
+                    }
                 }
             }
         } else if (ok) {
@@ -829,125 +1048,6 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     if (warp == C::MMA_WARP) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
-    }
-}
-
-struct PrefillMergeParams {
-    const int32_t* ctx_lens;
-    const int32_t* cu_q_lens;
-    const float* part_ml;
-    const float* part_o;
-    __nv_bfloat16* out;
-    int batch, max_blocks, total_q, H, tpg, split_steps, split_cap;
-};
-
-// Merge of the KV splits of pa_prefill_tc_kernel: one warp per (query token, head) row.
-//   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,   M = max_s m_s
-// over the splits the row's tile has visited.  Rows of sequences with a single split were
-// written by the attention kernel itself and are skipped, as are rows of refused sequences.
-template <int D>
-__global__ void __launch_bounds__(256) pa_prefill_merge_kernel(const PrefillMergeParams p) {
-    constexpr int NV = (D / 4 + 31) / 32;  // float4 pieces of a row per lane
-    pdl_launch_dependents();
-    // the lengths are inputs of the call, complete before the attention kernel let this grid
-    // start: the row's sequence and its number of splits are worked out while attention runs
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    int n_vis = 0;  // stays 0 for a row this kernel leaves alone
-    if (row < (long long)p.total_q * p.H) {
-        const int qi = (int)(row / p.H);
-        int lo = 0, hi = p.batch;  // last b with cu_q_lens[b] <= qi
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (__ldg(&p.cu_q_lens[mid]) <= qi) lo = mid; else hi = mid;
-        }
-        const int b = lo;
-        const int q0 = __ldg(&p.cu_q_lens[b]), q1 = __ldg(&p.cu_q_lens[b + 1]), L = __ldg(&p.ctx_lens[b]);
-        const int ql = q1 - q0;
-        const bool ok = q0 >= 0 && ql >= 0 && q1 <= p.total_q && L >= ql &&
-                        L <= p.max_blocks * BS && (b > 0 || q0 == 0) && qi >= q0 && qi < q1;
-        const int n_split = ok ? kv_splits(L, p.split_steps) : 1;
-        if (n_split > 1) {
-            // splits visited by the row's tile group: those that start at or before its last position
-            const int tok0 = (qi - q0) / p.tpg * p.tpg;
-            const int pos_max = L - ql + min(tok0 + p.tpg, ql) - 1;
-            n_vis = min(n_split, (pos_max / 64 + 1 + p.split_steps - 1) / p.split_steps);
-        }
-    }
-    // every thread waits before it leaves: the grid must not count as complete, and let the
-    // next kernel in the stream go, before the attention kernel has finished
-    pdl_wait();
-    if (n_vis == 0) return;
-    const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + (size_t)row * p.split_cap;
-    const float4* po = reinterpret_cast<const float4*>(p.part_o) + (size_t)row * p.split_cap * (D / 4);
-    // the usual case, two to four splits: every row of every split is requested before the
-    // first weight is known, so the (exponent, sum) pairs and the rows share one round trip
-    const bool few = n_vis <= 4;
-    float4 o[4][NV];
-#pragma unroll
-    for (int s = 0; s < 4; ++s)
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c = lane + 32 * v;
-            o[s][v] = few && s < n_vis && c < D / 4 ? po[(size_t)s * (D / 4) + c]
-                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    float M = -INFINITY;
-    bool bad = false;
-    for (int s = lane; s < n_vis; s += 32) {
-        const float2 v = ml[s];
-        M = fmaxf(M, v.x);
-        bad |= v.y < 0.f;
-    }
-    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    bad = __any_sync(0xffffffffu, bad);
-    float4 acc[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    float lsum = 0.f;
-    if (few) {
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            if (s >= n_vis) break;
-            const float2 v2 = ml[s];
-            const float w = v2.x == -INFINITY ? 0.f : ex2(v2.x - M);
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                acc[v].x = fmaf(w, o[s][v].x, acc[v].x);
-                acc[v].y = fmaf(w, o[s][v].y, acc[v].y);
-                acc[v].z = fmaf(w, o[s][v].z, acc[v].z);
-                acc[v].w = fmaf(w, o[s][v].w, acc[v].w);
-            }
-            lsum = fmaf(w, v2.y, lsum);
-        }
-    } else
-#pragma unroll 4
-    for (int s = 0; s < n_vis; ++s) {
-        const float2 v2 = ml[s];
-        const float w = v2.x == -INFINITY ? 0.f : ex2(v2.x - M);
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c = lane + 32 * v;
-            if (c < D / 4) {
-                const float4 o = po[(size_t)s * (D / 4) + c];
-                acc[v].x = fmaf(w, o.x, acc[v].x);
-                acc[v].y = fmaf(w, o.y, acc[v].y);
-                acc[v].z = fmaf(w, o.z, acc[v].z);
-                acc[v].w = fmaf(w, o.w, acc[v].w);
-            }
-        }
-        lsum = fmaf(w, v2.y, lsum);
-    }
-    const float inv = (bad || !(lsum > 0.f)) ? 0.f : 1.f / lsum;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int c = lane + 32 * v;
-        if (c < D / 4) {
-            uint2 w;
-            w.x = bad ? 0u : pack_bf16x2(acc[v].x * inv, acc[v].y * inv);
-            w.y = bad ? 0u : pack_bf16x2(acc[v].z * inv, acc[v].w * inv);
-            reinterpret_cast<uint2*>(p.out + (size_t)row * D)[c] = w;
-        }
     }
 }
 
@@ -1021,12 +1121,22 @@ static int launch_prefill_tc(const CUtensorMap& qm, const CUtensorMap& km, const
 
 using namespace pk;
 
-// The partial records follow the plan: first the (exponent, sum) pairs, then the fp32 rows, which
-// are written and read 16 bytes at a time.  An odd number of pairs would leave the rows 8-byte
-// aligned only, so the pair region is rounded up to 16 bytes and the workspace carries the pad.
-constexpr size_t PART_PAD_BYTES = 16;
-static size_t part_ml_floats(int64_t total_q, int H, int split_cap) {
-    return ((size_t)total_q * H * split_cap * 2 + 3) & ~(size_t)3;
+// After the plan come the arrival counters of the row groups (one int per row group and KV
+// head; the number of row groups is bounded with one tile per CTA) and the partial records of
+// the KV splits: whole 128-row tiles, so a chunk whose sequences end inside a tile, or whose
+// head group does not divide 128, holds more rows than it has queries.
+static size_t prefill_groups_bound(int64_t total_q, int64_t batch, int G, int Hkv) {
+    const int64_t tpt = 128 / G;
+    return (size_t)((total_q + tpt - 1) / tpt + batch + 1) * Hkv;
+}
+static size_t prefill_counter_bytes(int64_t total_q, int64_t batch, int G, int Hkv) {
+    return (prefill_groups_bound(total_q, batch, G, Hkv) * sizeof(int) + 255) & ~(size_t)255;
+}
+// bytes of the records of one split: every bounded row group as one tile of 128 rows, two for
+// the last group of each sequence when a CTA takes two tiles
+static size_t prefill_split_bytes(int64_t total_q, int64_t batch, int G, int Hkv, int D) {
+    const size_t tiles = prefill_groups_bound(total_q, batch, G, Hkv) + (size_t)(batch + 1) * Hkv;
+    return tiles * 128 * (size_t)(D + 2) * sizeof(float);
 }
 
 static size_t prefill_base_bytes(int64_t batch) {
@@ -1049,8 +1159,11 @@ extern "C" int pa_prefill_split_workspace_bytes(const pa_shape* shape, int32_t m
     int rc = validate_shape(shape);
     if (rc) return rc;
     if (max_batch < 0 || max_total_q < 0 || max_splits < 1) return PA_ERR_ARG;
-    *bytes = prefill_base_bytes(max_batch) + PART_PAD_BYTES +
-             (size_t)max_total_q * shape->num_q_heads * max_splits * (shape->head_dim + 2) * sizeof(float);
+    const int G = shape->num_q_heads / shape->num_kv_heads;
+    *bytes = prefill_base_bytes(max_batch) +
+             prefill_counter_bytes(max_total_q, max_batch, G, shape->num_kv_heads) +
+             (size_t)max_splits *
+                 prefill_split_bytes(max_total_q, max_batch, G, shape->num_kv_heads, shape->head_dim);
     return PA_OK;
 }
 
@@ -1105,7 +1218,12 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
             const bool even = r == T;
             double t = makespan(even ? groups * S : groups * (S - 1), T * step_us + unit_us,
                                 even ? 0 : groups, r * step_us + unit_us, sm_count);
-            if (S > 1) t += 6.0 + (double)total_q * H * S * (D + 2) * 4 * 2 / 5.0e6;
+            // a split unit writes its record and counts itself in (4.5 us measured); the last
+            // one of a row group then reads the other records of its tiles, about 25 us per MB
+            // (3.2 us per other split at head_dim 128 with two tiles), half as fast beyond
+            // four splits where its loads are not batched
+            if (S > 1)
+                t += 4.5 + (double)(S - 1) * nt * 128 * D * 4 * (S <= 4 ? 25e-6 : 50e-6);
             if (t < best_t) {
                 best_t = t;
                 best = {nt, S > 1 ? (int)T : 0, (int)std::max<int64_t>(S, 1)};
@@ -1129,6 +1247,31 @@ static TcShape choose_tc_shape(int64_t total_q, int batch, int Hkv, int G, int H
 }
 static thread_local TcShape g_last_shape = {0, 0, 1};
 
+// The number of this call among the calls with a KV split on `workspace` (1 .. 2^23 - 1, then
+// from 1 again): the arrival counters carry it, so that what an earlier call left in them
+// counts as zero.  `fresh`: the workspace is not in the table (oldest entry replaced first) or
+// its numbering starts over -- its counters may hold anything and are cleared.
+static int next_epoch(const void* workspace, bool* fresh) {
+    struct Entry {
+        const void* ws;
+        int epoch;
+    };
+    static std::mutex mu;
+    static Entry table[64] = {};
+    static int next = 0;
+    std::lock_guard<std::mutex> lk(mu);
+    for (Entry& e : table)
+        if (e.ws == workspace) {
+            e.epoch = e.epoch + 1 < (1 << 23) ? e.epoch + 1 : 1;
+            *fresh = e.epoch == 1;
+            return e.epoch;
+        }
+    table[next] = Entry{workspace, 1};
+    next = (next + 1) % 64;
+    *fresh = true;
+    return 1;
+}
+
 // What pa_prefill_split launches for these arguments (host arithmetic only).  tiles_per_cta 0
 // = the warp-level kernel.
 static int select_launch(const pa_shape* shape, int batch, int64_t total_q, int max_blocks_per_seq,
@@ -1149,10 +1292,10 @@ static int select_launch(const pa_shape* shape, int batch, int64_t total_q, int 
     *out = TcShape{0, 0, 1};
     if (force_mma) return PA_OK;
     const int64_t steps_bound = std::max<int64_t>(1, ((int64_t)max_blocks_per_seq * BS + 63) / 64);
-    const size_t per_split = (size_t)std::max<int64_t>(total_q, 1) * H * (D + 2) * sizeof(float);
-    const size_t part_bytes = workspace_bytes - base_bytes;
+    const size_t per_split = prefill_split_bytes(total_q, batch, G, shape->num_kv_heads, D);
+    const size_t fixed_bytes = base_bytes + prefill_counter_bytes(total_q, batch, G, shape->num_kv_heads);
     const int64_t cap_fit =
-        part_bytes > PART_PAD_BYTES ? (int64_t)((part_bytes - PART_PAD_BYTES) / per_split) : 0;
+        workspace_bytes > fixed_bytes ? (int64_t)((workspace_bytes - fixed_bytes) / per_split) : 0;
     int forced_steps = 0;
     if (kv_split_tokens > 0) {
         forced_steps = (kv_split_tokens + 63) / 64;
@@ -1293,43 +1436,31 @@ extern "C" int pa_prefill_split(const pa_shape* shape, const void* q, const void
         tp.split_cap = ts.split_cap;
         tp.fold_plan = fold_plan ? 1 : 0;
         tp.total_q = total_q;
-        tp.part_ml = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + base_bytes);
-        tp.part_o = tp.part_ml + part_ml_floats(total_q, H, ts.split_cap);
+        // counters, then the (exponent, sum) pairs of every record, then the rows
+        uint8_t* after_plan = static_cast<uint8_t*>(workspace) + base_bytes;
+        const size_t n_rec = (size_t)((total_q / plan.tpg + batch + 1) * pp.Hkv) * ts.split_cap *
+                             ts.tiles_per_cta;
+        tp.arrive = reinterpret_cast<int*>(after_plan);
+        tp.part_ml = reinterpret_cast<float*>(after_plan + prefill_counter_bytes(total_q, batch, G, pp.Hkv));
+        tp.part_o = tp.part_ml + n_rec * 128 * 2;
+        tp.epoch = 0;
+        if (ts.split_steps) {
+            bool fresh = false;
+            tp.epoch = next_epoch(workspace, &fresh);
+            if (fresh) {  // never seen (or long ago): no word may look like a count of this epoch
+                rc = check_cuda(cudaMemsetAsync(
+                    after_plan, 0, prefill_counter_bytes(total_q, batch, G, pp.Hkv), st));
+                if (rc) return rc;
+            }
+        }
         const int64_t max_ctas = ((int64_t)total_q / plan.tpg + batch) * pp.Hkv * ts.split_cap;
         if (max_ctas > INT32_MAX) return PA_ERR_ARG;
         const bool two = ts.tiles_per_cta == 2;
-        rc = D == 256  ? launch_prefill_tc<256, 1>(qm, km, vm, tp, (int)max_ctas, dev, st)
-             : D == 128 ? (two ? launch_prefill_tc<128, 2>(qm, km, vm, tp, (int)max_ctas, dev, st)
-                               : launch_prefill_tc<128, 1>(qm, km, vm, tp, (int)max_ctas, dev, st))
-                        : (two ? launch_prefill_tc<64, 2>(qm, km, vm, tp, (int)max_ctas, dev, st)
-                               : launch_prefill_tc<64, 1>(qm, km, vm, tp, (int)max_ctas, dev, st));
-        if (rc || ts.split_steps == 0) return rc;
-        PrefillMergeParams mp;
-        mp.ctx_lens = ctx_lens;
-        mp.cu_q_lens = cu_q_lens;
-        mp.part_ml = tp.part_ml;
-        mp.part_o = tp.part_o;
-        mp.out = pp.out;
-        mp.batch = batch;
-        mp.max_blocks = max_blocks_per_seq;
-        mp.total_q = total_q;
-        mp.H = H;
-        mp.tpg = plan.tpg;
-        mp.split_steps = ts.split_steps;
-        mp.split_cap = ts.split_cap;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(((int64_t)total_q * H + 7) / 8));
-        cfg.blockDim = dim3(256);
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        count_launch();
-        return check_cuda(D == 256   ? cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel<256>, mp)
-                          : D == 128 ? cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel<128>, mp)
-                                     : cudaLaunchKernelEx(&cfg, pa_prefill_merge_kernel<64>, mp));
+        return D == 256  ? launch_prefill_tc<256, 1>(qm, km, vm, tp, (int)max_ctas, dev, st)
+               : D == 128 ? (two ? launch_prefill_tc<128, 2>(qm, km, vm, tp, (int)max_ctas, dev, st)
+                                 : launch_prefill_tc<128, 1>(qm, km, vm, tp, (int)max_ctas, dev, st))
+                          : (two ? launch_prefill_tc<64, 2>(qm, km, vm, tp, (int)max_ctas, dev, st)
+                                 : launch_prefill_tc<64, 1>(qm, km, vm, tp, (int)max_ctas, dev, st));
     }
     return D == 256   ? launch_prefill<256>(km, vm, pp, dev, st)
            : D == 128 ? launch_prefill<128>(km, vm, pp, dev, st)

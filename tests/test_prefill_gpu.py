@@ -228,6 +228,39 @@ def test_forced_split_with_odd_head_count_and_odd_token_count(H, Hkv, D):
     assert_parity(out, ref, f"H{H}/{Hkv} D{D} odd split", amended=abs_ref)
 
 
+def test_split_calls_queued_on_one_workspace_keep_their_counts_apart():
+    """The units of a split call count themselves in per row group, in counters that live in
+    the workspace and carry the call's number.  Chunks of one growing context are queued on one
+    workspace without synchronisation (the recomputation pattern), with different split
+    lengths, and one chunk is repeated; every chunk's rows must match the oracle."""
+    H, Hkv, D = 32, 8, 128
+    L, chunk = 2304, 256
+    spec, q, k, v, _ = make_case([L], [L], H, Hkv, D, seed=91)
+    ref, abs_ref = prefill_ref(q, k, v, spec.block_tables, spec.seq_lens, np.array([0, L], np.int32),
+                               spec.scale)
+    g = GpuPrefill(spec, q, k, v, max_splits=40)
+    g.ws = torch.full((api.pa_prefill_split_workspace_bytes(api.shape_of(g.k, H), 1, chunk, 40) // 4,),
+                      float("nan"), dtype=torch.float32, device="cuda")
+    out = torch.full_like(g.q, float("nan"))
+    again = torch.full_like(g.q[:chunk], float("nan"))
+    splits = [0, 64, 512, 0, 128, 320, 64, 0, 1024]
+    for i, start in enumerate(range(0, L, chunk)):
+        end = start + chunk
+        args = (g.k, g.v, g.tables[:, :(end + 15) // 16].contiguous(),
+                torch.tensor([end], dtype=torch.int32, device="cuda"),
+                torch.tensor([0, chunk], dtype=torch.int32, device="cuda"), spec.scale)
+        api.pa_prefill_split(g.q[start:end], *args, out[start:end], g.ws,
+                             kv_split_tokens=splits[i], dev_status=g.status)
+        if start == 4 * chunk:  # the same chunk once more, into other rows
+            api.pa_prefill_split(g.q[start:end], *args, again, g.ws, kv_split_tokens=64,
+                                 dev_status=g.status)
+    torch.cuda.synchronize()
+    assert int(g.status.item()) == 0
+    assert_parity(torch_to_f64(out), ref, "queued split chunks", amended=abs_ref)
+    assert_parity(torch_to_f64(again), ref[4 * chunk:5 * chunk], "repeated chunk",
+                  amended=lambda: abs_ref()[4 * chunk:5 * chunk])
+
+
 def test_kv_split_with_two_tiles_per_cta():
     # enough query tokens for two row tiles per CTA; queries in the middle of the context, so
     # the first tiles end before the last splits begin
