@@ -2,8 +2,8 @@
 // sequence): every query token of the chunk attends to the cached tokens up to its own
 // position.  Two implementations behind pa_prefill / pa_prefill_split:
 //   * pa_prefill_tc_kernel: tcgen05 tensor cores, 128-row tiles, scores, weights and output
-//     accumulator in tensor memory, optionally the KV range of a tile split over CTAs with
-//     pa_prefill_merge_kernel combining the partial rows (every supported shape);
+//     accumulator in tensor memory, optionally the KV range of a tile split over CTAs, the
+//     last of which to finish combines the partial rows (every supported shape);
 //   * pa_prefill_kernel: the independent-warp machinery of decode -- a warp owns 16 query rows
 //     (tokens x heads of one KV-head group) and streams the KV blocks they may see through
 //     its private TMA ring; selected with PAGEDKV_PREFILL=mma, kept as a second implementation.
@@ -507,7 +507,7 @@ pa_prefill_tc_kernel(const __grid_constant__ CUtensorMap qmap,
     // misc[0] = TMEM base address, misc[1] = abort flag, misc[2] = bad block id seen,
     // misc[3] = this unit is the last of its row group to arrive
 
-    // Dependents (the merge kernel, the next call) start once every CTA here has passed the
+    // Dependents (the next call) start once every CTA here has passed the
     // wait, i.e. when all that precedes this call in the stream is complete: they may then read
     // the call's inputs before they wait for this grid themselves.
     pdl_wait();
